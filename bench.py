@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the MEDA compression pass (see the design doc for what is measured and how).
+
+One "step" = the whole pass (phase A of every layer, the budget barrier, phase B of every layer)
+over one synthetic prompt.  The metric is KV tokens compressed per second per layer-pass:
+    value = n_gpus * n_layers * n_tokens / step_time        [token*layers / s]
+With --gpus N > 1 (launched by torchrun) every rank compresses its own prompt (independent
+problems, no data-path collective): weak scaling.
+
+`--impl reference` times the CPU oracle (the only reference this paper has) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "kv_tokens_compressed_per_s_per_layer_pass"
+UNIT = "token*layers/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long_video_128k")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"], bf16_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample_seconds(wl, layer=0):
+    """Times the oracle, as it stands, on a bounded sample of the workload: one layer, KV head 0
+    with its query heads: scores + entropy of that head group, selection of that head at the uniform
+    budget rho * n, and merging of every `stride`-th less-important row (stride > 1 only for long
+    prompts; the merge time is multiplied back by the stride).  Returns (seconds, description)."""
+    import numpy as np
+    import torch
+    from oracle import meda_oracle as O
+    from paper_2502_17599_b200 import workloads as W
+
+    g = wl.n_q_heads // wl.n_kv_heads
+    sub = wl.with_(n_layers=max(layer + 1, 1))
+    q, k, v = W.make_layer(sub, layer, "cpu")
+    qh = q[:g].to(torch.float64).numpy()
+    kh = k[:1].to(torch.float64).numpy()
+    vh = v[:1].to(torch.float64).numpy()
+    mod = wl.modality().numpy()
+    s = max(wl.min_budget, int(round(wl.rho * wl.n_tokens)))
+    m = (s * 3) // 4
+    stride = max(1, wl.n_tokens // 16384)
+    t0 = time.perf_counter()
+    a_s = O.window_scores(qh, kh)
+    O.cross_modal_entropy(qh, kh, mod)
+    conserved, less = O.select_topk(a_s[0], mod, m, s - m)
+    t1 = time.perf_counter()
+    km, vm, counts, target = O.merge_kv(kh[0], vh[0], conserved, less[::stride])
+    O.round_to_dtype(km, wl.dtype), O.round_to_dtype(vm, wl.dtype)
+    t2 = time.perf_counter()
+    dt = (t1 - t0) + stride * (t2 - t1)
+    return dt, (f"layer {layer}, KV head 0 of {wl.n_kv_heads} ({g} query heads), uniform budget S={s}, merge on every "
+                f"{stride}-th less-important row with its time x{stride}; extrapolated x{wl.n_kv_heads} heads")
+
+
+def oracle_throughput(wl, seconds):
+    # one KV head of one layer took `seconds`: a whole layer-pass takes n_kv_heads times that
+    return wl.n_tokens / (seconds * wl.n_kv_heads)
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2502_17599_b200 import workloads as W
+    wl = W.WORKLOADS[args.workload]
+    import numpy  # noqa: F401  (loads BLAS before the thread count is read)
+    times = []
+    desc = ""
+    for i in range(args.warmup + args.steps):
+        dt, desc = oracle_sample_seconds(wl)
+        if i >= args.warmup:
+            times.append(dt)
+    sec = sum(times) / len(times)
+    val = oracle_throughput(wl, sec)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "shape": wl.description, "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# Clock sampling during the timed region
+# ------------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.rows = []
+        self.proc = None
+        self.index = device_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            p = [x.strip() for x in r.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0]))
+                smax.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, p[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# Our arm
+# ------------------------------------------------------------------------------------------------
+
+def algorithmic_work(wl, budgets):
+    """Algorithmic bytes / flops per layer-pass of each kernel class ('Roofline')."""
+    e = wl.element_size
+    n, d, hkv, hq, w = wl.n_tokens, wl.head_dim, wl.n_kv_heads, wl.n_q_heads, wl.window
+    kbytes = hkv * n * d * e
+    out = {"stats_bytes": [], "sweep_bytes": [], "nearest_flops": [], "reduce_bytes": []}
+    for s in budgets:
+        s = int(s)
+        out["stats_bytes"].append(kbytes)
+        out["sweep_bytes"].append(kbytes + 4 * hkv * n)
+        out["nearest_flops"].append(2.0 * (n - s) * s * d * hkv)
+        out["reduce_bytes"].append(2 * hkv * n * d * e + 2 * hkv * s * d * e + 4 * hkv * s)
+    return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_17599_b200 import build
+    from paper_2502_17599_b200 import workloads as W
+    from paper_2502_17599_b200.pipeline import CompressionPass
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    wl = W.WORKLOADS[args.workload].with_(seed=W.WORKLOADS[args.workload].seed + 1000 * rank)
+    L = wl.n_layers
+    qs, ks, vs = [], [], []
+    for l in range(L):
+        q, k, v = W.make_layer(wl, l, "cuda")
+        qs.append(q); ks.append(k); vs.append(v)
+    input_bytes = sum(t.numel() * t.element_size() for ts in (qs, ks, vs) for t in ts)
+    cp = CompressionPass(wl)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        cp.run(qs, ks, vs)
+    cp.ctx.check()
+    budgets = cp.budgets.cpu().numpy()[:, 0]
+
+    cp.ctx.profile_enable(True)
+    launches0 = cp.ctx.launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        cp.run(qs, ks, vs)
+    ev1.record(stream)
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = cp.ctx.launch_count() - launches0
+    prof = cp.ctx.profile_read()
+    cp.ctx.profile_enable(False)
+    cp.ctx.check()
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t[0]) / args.steps
+    value = world * L * wl.n_tokens / (ms_step * 1e-3)
+
+    # end-to-end leg: pinned host inputs -> device -> pass -> compacted caches back to the host
+    e2e = None
+    if not args.no_e2e:
+        q_h = [t_.cpu().pin_memory() for t_ in qs]
+        k_h = [t_.cpu().pin_memory() for t_ in ks]
+        v_h = [t_.cpu().pin_memory() for t_ in vs]
+        staging = {"q": qs, "k": ks, "v": vs}
+        out_host = cp.alloc_host_outputs()
+        h2d, d2h = cp.run_from_host(q_h, k_h, v_h, staging, out_host)      # warm-up
+        barrier()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            h2d, d2h = cp.run_from_host(q_h, k_h, v_h, staging, out_host)
+        e1.record(stream)
+        barrier()
+        wall = (time.perf_counter() - t0) * 1e3
+        ms_e2e = max(e0.elapsed_time(e1), wall) / args.e2e_steps
+        te = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * L * wl.n_tokens / (float(te[0]) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": float(te[0])}
+        del q_h, k_h, v_h, out_host
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    work = algorithmic_work(wl, budgets)
+    per_class = {name: {"ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps}
+                 for name, (ms, cnt) in prof.items() if cnt}
+    total_prof = sum(v["ms_per_step"] for v in per_class.values()) or 1.0
+    for v in per_class.values():
+        v["share"] = v["ms_per_step"] / total_prof
+    dominant = max(per_class, key=lambda k_: per_class[k_]["ms_per_step"])
+    # roofline of the dominant kernel
+    if dominant == "nearest":
+        flops = sum(work["nearest_flops"])
+        achieved = flops / (per_class["nearest"]["ms_per_step"] * 1e-3) / 1e12
+        roof = {"kernel": "nearest (merge similarity + arg-max)", "bound": "tensor", "achieved": achieved,
+                "peak": pk["bf16_sustained"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"],
+                "traffic": None, "peak_source": pk["source"] + " (sustained cuBLAS bf16)",
+                "flops_per_step": flops}
+    else:
+        key = {"stats": "stats_bytes", "sweep": "sweep_bytes", "reduce": "reduce_bytes"}.get(dominant)
+        nbytes = sum(work[key]) if key else 0.0
+        achieved = nbytes / (per_class[dominant]["ms_per_step"] * 1e-3) / 1e9 if key else 0.0
+        roof = {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"] + " (copy)",
+                "bytes_per_step": nbytes}
+    # secondary fractions, for the record
+    extra = {}
+    for name, key in (("stats", "stats_bytes"), ("sweep", "sweep_bytes"), ("reduce", "reduce_bytes")):
+        if name in per_class:
+            gbs = sum(work[key]) / (per_class[name]["ms_per_step"] * 1e-3) / 1e9
+            extra[name] = {"GB/s": gbs, "frac_of_copy_peak": gbs / pk["hbm_gbs"]}
+    if "nearest" in per_class:
+        tf = sum(work["nearest_flops"]) / (per_class["nearest"]["ms_per_step"] * 1e-3) / 1e12
+        extra["nearest"] = {"TFLOP/s": tf, "frac_of_sustained_bf16": tf / pk["bf16_sustained"]}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        sec, desc = oracle_sample_seconds(W.WORKLOADS[args.workload])
+        cpu = {"value": oracle_throughput(wl, sec), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+               "sample": desc, "sample_seconds": sec}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "shape": wl.description, "global_budget": wl.global_budget,
+                   "input_bytes": input_bytes, "l2": "inputs larger than L2 (no flush needed)" if input_bytes > 256e6 else "inputs fit L2",
+                   "parallelism": f"independent prompts x{world}"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roof, "kernels": per_class, "kernel_rooflines": extra, "cpu_baseline": cpu,
+        "budgets_min_max": [int(budgets.min()), int(budgets.max())],
+    }
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,198 @@
+/*
+ * meda.h - C ABI of the B200-native MEDA prefill KV-cache compression pass
+ * (MEDA: "Dynamic KV Cache Allocation for Efficient Multimodal Long-Context Inference",
+ *  arXiv 2502.17599, Sections 3.2-3.3 and 4.4, Appendix A.3).
+ *
+ * The pass runs once after prompt encoding and before decoding:
+ *   phase A, per layer : attention of an observation window of text queries against the whole
+ *                        key cache -> per-key accumulated scores (Eq. 8) and the cross-modal
+ *                        attention entropy E_CM of the layer (Eq. 4-6);
+ *   barrier            : softmax over all layers' entropies -> integer per-layer budgets that sum
+ *                        to the global budget (Eq. 7), each split recent : important;
+ *   phase B, per layer : per KV head, keep the recent tokens plus the top-scoring ones with text
+ *                        first (Eq. 9-10); merge every other KV pair into its most cosine-similar
+ *                        kept key by averaging (Eq. 11-12).
+ *
+ * Conventions that hold for every entry point unless it says otherwise
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller; the library neither frees it
+ *    nor keeps it after the call's work has run.  `spans_host` and `meda_config` are HOST memory.
+ *  - Layouts are dense and row-major: caches [n_kv_heads][n_tokens][head_dim], query windows
+ *    [n_q_heads][window][head_dim], element type `dtype` (bf16 or fp32).  Query head h belongs
+ *    to KV head h / (n_q_heads / n_kv_heads).  Window row i is the token at absolute position
+ *    n_tokens - window + i and, as in decoder prefill, sees keys j <= that position.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue
+ *    work and return; nothing is copied back to the host between steps.
+ *  - Step calls allocate nothing: all scratch memory is taken from the context at meda_create.
+ *    A context may be used by one host thread and one stream at a time.
+ *  - Errors the host can see (NULL pointers, bad shapes, bad layer index) return a negative
+ *    status before anything is launched.  Errors only the device can see (a budget row that does
+ *    not fit `out_capacity`, a bounded wait that ran out) are recorded in a status word that
+ *    meda_poll_status returns; the kernel that saw the error skips its work and returns.
+ *  - `budgets` is int32 [n_layers][3] = (S_l, M_l, N_l): conserved rows, recent rows, top-scored
+ *    rows (S_l = M_l + N_l).  It stays on the device; kernels read their layer's row.
+ */
+#ifndef MEDA_H_
+#define MEDA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct meda_ctx meda_ctx; /* opaque: configuration, modality map and scratch memory */
+
+typedef enum {
+  MEDA_OK = 0,
+  MEDA_ERR_INVALID_ARG = -1,       /* NULL pointer, bad enum, layer out of range */
+  MEDA_ERR_SHAPE = -2,             /* sizes the kernels do not support or that contradict each other */
+  MEDA_ERR_BUDGET_INFEASIBLE = -3, /* global budget outside [L*min_budget, L*n_tokens] */
+  MEDA_ERR_WORKSPACE = -4,         /* an output capacity is too small for the layer's budget */
+  MEDA_ERR_CUDA = -5,              /* a CUDA runtime call failed */
+  MEDA_ERR_UNSUPPORTED = -6,       /* valid request that this build does not implement */
+  MEDA_ERR_TIMEOUT = -7            /* a bounded device-side wait ran out */
+} meda_status;
+
+typedef enum { MEDA_BF16 = 0, MEDA_F32 = 1 } meda_dtype;
+enum { MEDA_TEXT = 0, MEDA_VISUAL = 1 };
+
+/* One run of tokens of a single modality, [begin, end).  The table passed to meda_create must be
+ * sorted, disjoint and cover [0, n_tokens) exactly (Sec. 3.1: the prompt is an interleaving of
+ * text and image / video token runs; Sec. 3.2 splits Q and K "based on the modality index"). */
+typedef struct {
+  int32_t begin, end, modality;
+} meda_span;
+
+typedef struct {
+  int32_t n_layers, n_q_heads, n_kv_heads, head_dim, n_tokens, window;
+  int32_t dtype;          /* meda_dtype of caches, query windows and outputs */
+  int64_t global_budget;  /* B = sum_l S_l in token*layers; Eq. 7 with B = round(rho * L * n_tokens) */
+  int32_t beta_recent;    /* recent : important split of each layer budget, 3 : 1 in Sec. 4.4 */
+  int32_t beta_important;
+  int32_t min_budget;     /* per-layer floor of S_l (>= 1); n_tokens is the ceiling */
+  int32_t entropy_mode;   /* 0: entropy of the head-averaged attention (Sec. 3.2); 1: mean of per-head entropies */
+  int32_t alloc_mode;     /* 0: Eq. 7; 1: uniform shares (Table 5, "w/o dynamic allocation") */
+  int32_t merge_mode;     /* 0: Eq. 12 average merging; 1: drop the less important pairs (Table 5, "w/o merging") */
+} meda_config;
+
+/* Creates a context: validates the configuration, uploads the modality map built from
+ * `spans_host` (host memory, n_spans entries) and allocates all scratch memory on the current
+ * device (the only allocating call).  Supported shapes: head_dim in {64, 128, 256} for fp32 and
+ * bf16, n_q_heads a multiple of n_kv_heads, 1 <= window <= min(n_tokens, 128), n_layers <= 1024.
+ * On failure *out is NULL and the status says why. */
+meda_status meda_create(const meda_config* config, const meda_span* spans_host, int32_t n_spans, meda_ctx** out);
+
+/* Frees the context's scratch memory.  The caller must have synchronised the streams that used it. */
+void meda_destroy(meda_ctx* ctx);
+
+/* Static, NUL-terminated description of a status code. */
+const char* meda_status_string(meda_status status);
+
+/* Bytes of device scratch memory the context holds. */
+int64_t meda_workspace_bytes(const meda_ctx* ctx);
+
+/* Synchronises `stream`, returns the first device-side error recorded since the last poll (or
+ * MEDA_OK) and clears it. */
+meda_status meda_poll_status(meda_ctx* ctx, void* stream);
+
+/* Phase A, one layer (Eq. 4 and Eq. 8 with the query rows restricted to the observation window).
+ * Two sweeps over the key cache.  The first computes every window row's softmax normalisers:
+ *   row_stats fp32 [n_q_heads][window][4] = (max, sum exp(s - max)) over all visible keys and
+ *   (max, sum exp) over the visible VISUAL keys, s = q.k / sqrt(head_dim); a row that sees no
+ *   visual key has (-inf, 0) there.
+ * The second computes the per-key accumulated attention
+ *   scores fp32 [n_kv_heads][n_tokens]: A_s[g][j] = sum over window rows i and query heads h of
+ *   KV head g of softmax_j(s)[h][i][j]   (each KV head's scores sum to group_size * window)
+ * and, when `entropy` is not NULL, in the same sweep the layer's cross-modal entropy
+ *   entropy[layer] (fp32, device array of n_layers): E_CM = -E_TV of Eq. 5-6, the mean over
+ *   window rows of the entropy (natural log) of text-to-vision attention, whose softmax is taken
+ *   over the visual keys only; averaged over heads before or after the entropy per entropy_mode.
+ * q_win, k: device, `dtype`.  row_stats, scores: device outputs, fully overwritten. */
+meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                               float* row_stats, float* scores, float* entropy, void* stream);
+
+/* Cross-modal attention entropy of one layer from existing row_stats (Eq. 4-6): one sweep over
+ * the key cache, writes entropy[layer].  For callers that already hold the normalisers.
+ * q_vis / q_vis_pos / n_vis_rows describe an optional window of VISUAL query rows
+ * ([n_q_heads][n_vis_rows][head_dim] and their absolute positions) for the E_VT term of Eq. 5;
+ * pass NULL, NULL, 0 for the text-window-only definition E_CM = -E_TV.  A non-NULL q_vis
+ * returns MEDA_ERR_UNSUPPORTED in this build. */
+meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                               const float* row_stats, const void* q_vis, const int32_t* q_vis_pos,
+                               int32_t n_vis_rows, float* entropy, void* stream);
+
+/* Barrier step (Eq. 7, Appendix A.3, and Sec. 4.4 for the split): one thread block.
+ * weights W_l = softmax_l(entropy); real quotas q_l = clip(lambda W_l, min_budget, n_tokens) with
+ * lambda such that sum q_l = global_budget; S_l = floor(q_l) and the missing units go one each to
+ * the unclamped layers by largest fractional part, ties to the lowest layer;
+ * M_l = floor(S_l * beta_recent / (beta_recent + beta_important)), N_l = S_l - M_l.
+ * entropy: device fp32 [n_layers].  budgets: device int32 [n_layers][3], overwritten. */
+meda_status meda_allocate_budgets(meda_ctx* ctx, const float* entropy, int32_t* budgets, void* stream);
+
+/* Phase B, selection for one layer and all its KV heads (Eq. 9-10).  Candidates are tokens
+ * [0, n_tokens - M_l); they are ranked text before visual (Eq. 9's boost), then by score
+ * descending, then by index ascending; the first N_l are kept together with the last M_l tokens.
+ *   idx_conserved int32 [n_kv_heads][out_capacity]: the S_l kept token indices, ascending
+ *   idx_less      int32 [n_kv_heads][n_tokens]    : the n_tokens - S_l others, ascending
+ * Entries past those counts are left untouched.  S_l > out_capacity records MEDA_ERR_WORKSPACE. */
+meda_status meda_select_topk(meda_ctx* ctx, int32_t layer, const float* scores, const int32_t* budgets,
+                             int32_t* idx_conserved, int32_t* idx_less, int32_t out_capacity, void* stream);
+
+/* Phase B, merging for one layer and all its KV heads (Eq. 11-12).  For every less important
+ * token i the kept slot with the largest cosine similarity of keys, u = k_i.k_j / (|k_i||k_j|)
+ * with each norm clamped below at 1e-8, first maximum in slot order; then for keys and values
+ *   x_out[g][s] = (x[c_s] + sum of x[i] over tokens i assigned to s) / counts[g][s],
+ * sums over the ORIGINAL rows, accumulated in fp32 in ascending token order, rounded once to
+ * `dtype`.  With merge_mode 1 the kept rows are copied and counts are 1.
+ *   k_out, v_out `dtype` [n_kv_heads][out_capacity][head_dim]; counts int32 [n_kv_heads][out_capacity]
+ *   target int32 [n_kv_heads][n_tokens], optional (may be NULL): slot chosen for idx_less[g][p]
+ * Rows past S_l are left untouched. */
+meda_status meda_merge_kv(meda_ctx* ctx, int32_t layer, const void* k, const void* v, const int32_t* budgets,
+                          const int32_t* idx_conserved, const int32_t* idx_less,
+                          void* k_out, void* v_out, int32_t* counts, int32_t* target,
+                          int32_t out_capacity, void* stream);
+
+/* Phase B for one layer: meda_select_topk followed by meda_merge_kv, with the less-important
+ * list kept in the context's scratch memory (Sec. 3.3 as a whole). */
+meda_status meda_compress_layer(meda_ctx* ctx, int32_t layer, const void* k, const void* v, const float* scores,
+                                const int32_t* budgets, void* k_out, void* v_out, int32_t* counts,
+                                int32_t* idx_conserved, int32_t out_capacity, void* stream);
+
+/* ---- measurement helpers (no counterpart in the paper) ------------------------------------ */
+
+/* Kernel classes the library reports times for. */
+enum {
+  MEDA_K_STATS = 0,      /* phase A sweep 1: softmax normalisers */
+  MEDA_K_STATS_COMBINE,  /* merge of the partial normalisers */
+  MEDA_K_SWEEP,          /* phase A sweep 2: scores and/or entropy */
+  MEDA_K_ENTROPY_FINAL,  /* reduction of the entropy partials */
+  MEDA_K_ALLOCATE,       /* budgets */
+  MEDA_K_SELECT,         /* radix select + compaction */
+  MEDA_K_PREP,           /* conserved-key gather and inverse norms */
+  MEDA_K_NEAREST,        /* similarity contraction + arg-max */
+  MEDA_K_GROUP,          /* grouping of the less-important rows by target slot */
+  MEDA_K_REDUCE,         /* segmented average */
+  MEDA_K_CLASSES
+};
+
+/* Name of a kernel class ("stats", "sweep", ...), or NULL if out of range. */
+const char* meda_kernel_class_name(int32_t kernel_class);
+
+/* Turns per-launch timing on (enable != 0) or off.  Turning it on creates a pool of CUDA events
+ * (an allocating call: do it outside timed regions); while on, every kernel launch of a step call
+ * is bracketed by two events on the call's stream, up to the pool size, after which launches are
+ * still counted but no longer timed. */
+meda_status meda_profile_enable(meda_ctx* ctx, int32_t enable);
+
+/* Synchronises the recorded events and writes, per kernel class, the summed device time in
+ * milliseconds (ms_out, HOST float[MEDA_K_CLASSES]) and the number of timed launches
+ * (launches_out, HOST int32[MEDA_K_CLASSES]); then clears the record.  Either pointer may be NULL. */
+meda_status meda_profile_read(meda_ctx* ctx, float* ms_out, int32_t* launches_out);
+
+/* Number of kernels this context has launched since it was created (timing on or off). */
+int64_t meda_launch_count(const meda_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MEDA_H_ */

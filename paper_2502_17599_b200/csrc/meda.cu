@@ -1,0 +1,400 @@
+// C-ABI entry points of the MEDA compression pass (declared in include/meda.h): argument checks,
+// context and scratch memory, and kernel launches.  Host code here only enqueues work.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "allocate.cuh"
+#include "attn_generic.cuh"
+#include "meda_common.cuh"
+#include "merge_generic.cuh"
+#include "select.cuh"
+
+using namespace meda;
+
+namespace {
+
+constexpr int kMaxDynSmem = 227 * 1024;
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+#define MEDA_CUDA_TRY(expr)                         \
+  do {                                              \
+    cudaError_t e__ = (expr);                       \
+    if (e__ != cudaSuccess) return MEDA_ERR_CUDA;   \
+  } while (0)
+
+inline meda_status launch_status() { return cudaGetLastError() == cudaSuccess ? MEDA_OK : MEDA_ERR_CUDA; }
+
+template <typename T>
+meda_status carve(T** p, int64_t count, int64_t* total) {
+  int64_t bytes = ((count * (int64_t)sizeof(T)) + 255) / 256 * 256;
+  if (bytes == 0) bytes = 256;
+  if (cudaMalloc(reinterpret_cast<void**>(p), (size_t)bytes) != cudaSuccess) return MEDA_ERR_CUDA;
+  *total += bytes;
+  return MEDA_OK;
+}
+
+void free_workspace(Workspace& ws) {
+  cudaFree(ws.modality);
+  cudaFree(ws.status);
+  cudaFree(ws.stats_partial);
+  cudaFree(ws.ent_partial);
+  cudaFree(ws.inv_norm);
+  cudaFree(ws.target);
+  cudaFree(ws.idx_less);
+  ws = Workspace();
+}
+
+int generic_tiles(int n) { return (n + kGenericKeyTile - 1) / kGenericKeyTile; }
+
+template <typename T>
+meda_status set_generic_attrs(int stats_smem, int sweep_smem, int nn_smem) {
+  MEDA_CUDA_TRY(cudaFuncSetAttribute(stats_partial_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, stats_smem));
+  MEDA_CUDA_TRY(cudaFuncSetAttribute(scores_entropy_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, sweep_smem));
+  MEDA_CUDA_TRY(cudaFuncSetAttribute(nearest_generic_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, nn_smem));
+  return MEDA_OK;
+}
+
+// Brackets one kernel launch with profiling events (when enabled) and counts it.
+struct LaunchScope {
+  meda_ctx* ctx;
+  cudaStream_t st;
+  int slot = -1;
+  LaunchScope(meda_ctx* c, int klass, cudaStream_t s) : ctx(c), st(s) {
+    ++ctx->launches;
+    Profiler& p = ctx->prof;
+    if (p.enabled && p.used < Profiler::kPool) {
+      slot = p.used++;
+      p.klass[slot] = klass;
+      cudaEventRecord(p.begin[slot], st);
+    }
+  }
+  ~LaunchScope() {
+    if (slot >= 0) cudaEventRecord(ctx->prof.end[slot], st);
+  }
+};
+
+void profiler_release(Profiler& p) {
+  if (p.begin) {
+    for (int i = 0; i < Profiler::kPool; ++i) {
+      if (p.begin[i]) cudaEventDestroy(p.begin[i]);
+      if (p.end[i]) cudaEventDestroy(p.end[i]);
+    }
+  }
+  free(p.begin);
+  free(p.end);
+  free(p.klass);
+  p = Profiler();
+}
+
+bool layer_ok(const meda_ctx* ctx, int32_t layer) { return ctx && layer >= 0 && layer < ctx->cfg.n_layers; }
+
+// ---- phase A launches ------------------------------------------------------------------------
+template <typename T>
+meda_status launch_stats(meda_ctx* ctx, const void* q_win, const void* k, float* row_stats, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const float scale = 1.0f / sqrtf((float)c.head_dim);
+  const int chunks = std::min(kStatsChunks, generic_tiles(c.n_tokens));
+  const int smem = attn_generic_smem(c.window, c.head_dim, false).total;
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS, st);
+    stats_partial_kernel<T><<<dim3(chunks, c.n_q_heads), kAttnThreads, smem, st>>>(
+        static_cast<const T*>(q_win), static_cast<const T*>(k), ctx->ws.modality, ctx->ws.stats_partial,
+        c.n_q_heads, ctx->group, c.n_tokens, c.window, c.head_dim, scale);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
+    stats_combine_kernel<<<c.n_q_heads, kMaxWindow, 0, st>>>(ctx->ws.stats_partial, row_stats, chunks, c.n_q_heads, c.window);
+  }
+  return launch_status();
+}
+
+template <typename T>
+meda_status launch_sweep(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
+                         float* scores, float* entropy, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const float scale = 1.0f / sqrtf((float)c.head_dim);
+  const int tiles = generic_tiles(c.n_tokens);
+  const int smem = attn_generic_smem(c.window, c.head_dim, true).total;
+  {
+    LaunchScope scope(ctx, MEDA_K_SWEEP, st);
+    scores_entropy_kernel<T><<<tiles, kAttnThreads, smem, st>>>(
+        static_cast<const T*>(q_win), static_cast<const T*>(k), ctx->ws.modality, row_stats, scores,
+        ctx->ws.ent_partial, c.n_q_heads, ctx->group, c.n_tokens, c.window, c.head_dim, scale, c.entropy_mode,
+        scores != nullptr, entropy != nullptr);
+  }
+  if (entropy) {
+    LaunchScope scope(ctx, MEDA_K_ENTROPY_FINAL, st);
+    entropy_finalize_kernel<<<1, 256, 0, st>>>(ctx->ws.ent_partial, tiles, row_stats, c.window, entropy + layer);
+  }
+  return launch_status();
+}
+
+// ---- phase B launches ------------------------------------------------------------------------
+template <typename T>
+meda_status launch_merge(meda_ctx* ctx, const void* k, const void* v, const int32_t* budget_row,
+                         const int32_t* idx_conserved, const int32_t* idx_less, void* k_out, void* v_out,
+                         int32_t* counts, int32_t* target, int32_t cap, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const int n = c.n_tokens, d = c.head_dim;
+  const int max_slots = std::min(cap, n);
+  const int evict = c.merge_mode == 1;
+  if (!evict) {
+    {
+      LaunchScope scope(ctx, MEDA_K_PREP, st);
+      conserved_inv_norm_kernel<T><<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
+          static_cast<const T*>(k), idx_conserved, budget_row, ctx->ws.inv_norm, n, d, cap);
+    }
+    const int nn_smem = (kNnTile * (d + 1) + kNnTile * (kNnDk + 1)) * 4;
+    LaunchScope scope(ctx, MEDA_K_NEAREST, st);
+    nearest_generic_kernel<T><<<dim3((n + kNnTile - 1) / kNnTile, c.n_kv_heads), 256, nn_smem, st>>>(
+        static_cast<const T*>(k), idx_conserved, idx_less, budget_row, ctx->ws.inv_norm, target, n, d, cap);
+  }
+  LaunchScope scope(ctx, MEDA_K_REDUCE, st);
+  merge_scan_kernel<T><<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
+      static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, idx_less, target, budget_row,
+      static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n, d, cap, evict);
+  return launch_status();
+}
+
+}  // namespace
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+const char* meda_status_string(meda_status status) {
+  switch (status) {
+    case MEDA_OK: return "ok";
+    case MEDA_ERR_INVALID_ARG: return "invalid argument";
+    case MEDA_ERR_SHAPE: return "unsupported or inconsistent shape";
+    case MEDA_ERR_BUDGET_INFEASIBLE: return "budget infeasible";
+    case MEDA_ERR_WORKSPACE: return "output capacity too small";
+    case MEDA_ERR_CUDA: return "CUDA runtime error";
+    case MEDA_ERR_UNSUPPORTED: return "not implemented in this build";
+    case MEDA_ERR_TIMEOUT: return "bounded device wait ran out";
+  }
+  return "unknown status";
+}
+
+meda_status meda_create(const meda_config* config, const meda_span* spans_host, int32_t n_spans, meda_ctx** out) {
+  if (out) *out = nullptr;
+  if (!config || !spans_host || !out || n_spans <= 0) return MEDA_ERR_INVALID_ARG;
+  const meda_config& c = *config;
+  if (c.dtype != MEDA_BF16 && c.dtype != MEDA_F32) return MEDA_ERR_INVALID_ARG;
+  if (c.entropy_mode < 0 || c.entropy_mode > 1 || c.alloc_mode < 0 || c.alloc_mode > 1 || c.merge_mode < 0 ||
+      c.merge_mode > 1)
+    return MEDA_ERR_INVALID_ARG;
+  if (c.n_layers < 1 || c.n_layers > kMaxLayers || c.n_q_heads < 1 || c.n_kv_heads < 1 ||
+      c.n_q_heads % c.n_kv_heads != 0 || c.n_tokens < 1 || c.window < 1 || c.window > c.n_tokens ||
+      c.window > kMaxWindow)
+    return MEDA_ERR_SHAPE;
+  if (c.head_dim != 64 && c.head_dim != 128 && c.head_dim != 256) return MEDA_ERR_SHAPE;
+  if (c.beta_recent < 0 || c.beta_important < 0 || c.beta_recent + c.beta_important <= 0) return MEDA_ERR_INVALID_ARG;
+  if (c.min_budget < 1 || c.min_budget > c.n_tokens) return MEDA_ERR_BUDGET_INFEASIBLE;
+  if (c.global_budget < (int64_t)c.n_layers * c.min_budget || c.global_budget > (int64_t)c.n_layers * c.n_tokens)
+    return MEDA_ERR_BUDGET_INFEASIBLE;
+  if (attn_generic_smem(c.window, c.head_dim, true).total > kMaxDynSmem) return MEDA_ERR_SHAPE;
+
+  // modality map from the span table: sorted, disjoint, covering [0, n)
+  std::vector<uint8_t> modality((size_t)c.n_tokens);
+  int32_t pos = 0, n_visual = 0;
+  for (int32_t s = 0; s < n_spans; ++s) {
+    const meda_span& sp = spans_host[s];
+    if (sp.begin != pos || sp.end <= sp.begin || sp.end > c.n_tokens) return MEDA_ERR_INVALID_ARG;
+    if (sp.modality != MEDA_TEXT && sp.modality != MEDA_VISUAL) return MEDA_ERR_INVALID_ARG;
+    for (int32_t j = sp.begin; j < sp.end; ++j) modality[(size_t)j] = (uint8_t)sp.modality;
+    if (sp.modality == MEDA_VISUAL) n_visual += sp.end - sp.begin;
+    pos = sp.end;
+  }
+  if (pos != c.n_tokens) return MEDA_ERR_INVALID_ARG;
+
+  meda_ctx* ctx = new (std::nothrow) meda_ctx();
+  if (!ctx) return MEDA_ERR_CUDA;
+  ctx->cfg = c;
+  ctx->group = c.n_q_heads / c.n_kv_heads;
+  ctx->n_visual = n_visual;
+  if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess) {
+    delete ctx;
+    return MEDA_ERR_CUDA;
+  }
+  ctx->ent_slots = generic_tiles(c.n_tokens);
+
+  Workspace& ws = ctx->ws;
+  const int64_t n = c.n_tokens, hkv = c.n_kv_heads;
+  meda_status st = MEDA_OK;
+  if (st == MEDA_OK) st = carve(&ws.modality, n, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.status, 1, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.stats_partial, (int64_t)kStatsChunks * c.n_q_heads * c.window * 4, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.inv_norm, hkv * n, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.target, hkv * n, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.idx_less, hkv * n, &ws.bytes);
+  if (st == MEDA_OK && cudaMemcpy(ws.modality, modality.data(), (size_t)n, cudaMemcpyHostToDevice) != cudaSuccess)
+    st = MEDA_ERR_CUDA;
+  if (st == MEDA_OK && cudaMemset(ws.status, 0, sizeof(int)) != cudaSuccess) st = MEDA_ERR_CUDA;
+  if (st == MEDA_OK) {
+    const int stats_smem = attn_generic_smem(c.window, c.head_dim, false).total;
+    const int sweep_smem = attn_generic_smem(c.window, c.head_dim, true).total;
+    const int nn_smem = (kNnTile * (c.head_dim + 1) + kNnTile * (kNnDk + 1)) * 4;
+    st = c.dtype == MEDA_F32 ? set_generic_attrs<float>(stats_smem, sweep_smem, nn_smem)
+                             : set_generic_attrs<__nv_bfloat16>(stats_smem, sweep_smem, nn_smem);
+  }
+  if (st != MEDA_OK) {
+    free_workspace(ws);
+    delete ctx;
+    cudaGetLastError();
+    return st;
+  }
+  *out = ctx;
+  return MEDA_OK;
+}
+
+void meda_destroy(meda_ctx* ctx) {
+  if (!ctx) return;
+  profiler_release(ctx->prof);
+  free_workspace(ctx->ws);
+  delete ctx;
+}
+
+int64_t meda_workspace_bytes(const meda_ctx* ctx) { return ctx ? ctx->ws.bytes : 0; }
+
+int64_t meda_launch_count(const meda_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* meda_kernel_class_name(int32_t kernel_class) {
+  static const char* const names[MEDA_K_CLASSES] = {"stats", "stats_combine", "sweep", "entropy_final", "allocate",
+                                                    "select", "prep", "nearest", "group", "reduce"};
+  return kernel_class >= 0 && kernel_class < MEDA_K_CLASSES ? names[kernel_class] : nullptr;
+}
+
+meda_status meda_profile_enable(meda_ctx* ctx, int32_t enable) {
+  if (!ctx) return MEDA_ERR_INVALID_ARG;
+  Profiler& p = ctx->prof;
+  if (!enable) {
+    p.enabled = false;
+    return MEDA_OK;
+  }
+  if (!p.begin) {
+    p.begin = static_cast<cudaEvent_t*>(calloc(Profiler::kPool, sizeof(cudaEvent_t)));
+    p.end = static_cast<cudaEvent_t*>(calloc(Profiler::kPool, sizeof(cudaEvent_t)));
+    p.klass = static_cast<int*>(calloc(Profiler::kPool, sizeof(int)));
+    if (!p.begin || !p.end || !p.klass) { profiler_release(p); return MEDA_ERR_CUDA; }
+    for (int i = 0; i < Profiler::kPool; ++i) {
+      if (cudaEventCreate(&p.begin[i]) != cudaSuccess || cudaEventCreate(&p.end[i]) != cudaSuccess) {
+        profiler_release(p);
+        return MEDA_ERR_CUDA;
+      }
+    }
+  }
+  p.used = 0;
+  p.enabled = true;
+  return MEDA_OK;
+}
+
+meda_status meda_profile_read(meda_ctx* ctx, float* ms_out, int32_t* launches_out) {
+  if (!ctx) return MEDA_ERR_INVALID_ARG;
+  Profiler& p = ctx->prof;
+  float ms[MEDA_K_CLASSES] = {0};
+  int32_t cnt[MEDA_K_CLASSES] = {0};
+  for (int i = 0; i < p.used; ++i) {
+    MEDA_CUDA_TRY(cudaEventSynchronize(p.end[i]));
+    float t = 0.f;
+    MEDA_CUDA_TRY(cudaEventElapsedTime(&t, p.begin[i], p.end[i]));
+    ms[p.klass[i]] += t;
+    cnt[p.klass[i]] += 1;
+  }
+  p.used = 0;
+  if (ms_out) memcpy(ms_out, ms, sizeof(ms));
+  if (launches_out) memcpy(launches_out, cnt, sizeof(cnt));
+  return MEDA_OK;
+}
+
+meda_status meda_poll_status(meda_ctx* ctx, void* stream) {
+  if (!ctx) return MEDA_ERR_INVALID_ARG;
+  int code = 0;
+  MEDA_CUDA_TRY(cudaStreamSynchronize(as_stream(stream)));
+  MEDA_CUDA_TRY(cudaMemcpy(&code, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (code != 0) MEDA_CUDA_TRY(cudaMemset(ctx->ws.status, 0, sizeof(int)));
+  return (meda_status)code;
+}
+
+meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, float* row_stats,
+                               float* scores, float* entropy, void* stream) {
+  if (!layer_ok(ctx, layer) || !q_win || !k || !row_stats || !scores) return MEDA_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  meda_status r;
+  if (ctx->cfg.dtype == MEDA_F32) {
+    r = launch_stats<float>(ctx, q_win, k, row_stats, st);
+    if (r == MEDA_OK) r = launch_sweep<float>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+  } else {
+    r = launch_stats<__nv_bfloat16>(ctx, q_win, k, row_stats, st);
+    if (r == MEDA_OK) r = launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+  }
+  return r;
+}
+
+meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
+                               const void* q_vis, const int32_t* q_vis_pos, int32_t n_vis_rows, float* entropy,
+                               void* stream) {
+  if (!layer_ok(ctx, layer) || !q_win || !k || !row_stats || !entropy) return MEDA_ERR_INVALID_ARG;
+  if (q_vis || q_vis_pos || n_vis_rows != 0) return MEDA_ERR_UNSUPPORTED;
+  cudaStream_t st = as_stream(stream);
+  if (ctx->cfg.dtype == MEDA_F32) return launch_sweep<float>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
+  return launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
+}
+
+meda_status meda_allocate_budgets(meda_ctx* ctx, const float* entropy, int32_t* budgets, void* stream) {
+  if (!ctx || !entropy || !budgets) return MEDA_ERR_INVALID_ARG;
+  const meda_config& c = ctx->cfg;
+  LaunchScope scope(ctx, MEDA_K_ALLOCATE, as_stream(stream));
+  allocate_budgets_kernel<<<1, 32, 0, as_stream(stream)>>>(entropy, budgets, c.n_layers, (long long)c.global_budget,
+                                                           c.min_budget, c.n_tokens, c.beta_recent, c.beta_important,
+                                                           c.alloc_mode, ctx->ws.status);
+  return launch_status();
+}
+
+meda_status meda_select_topk(meda_ctx* ctx, int32_t layer, const float* scores, const int32_t* budgets,
+                             int32_t* idx_conserved, int32_t* idx_less, int32_t out_capacity, void* stream) {
+  if (!layer_ok(ctx, layer) || !scores || !budgets || !idx_conserved || !idx_less) return MEDA_ERR_INVALID_ARG;
+  if (out_capacity < 1) return MEDA_ERR_WORKSPACE;
+  const meda_config& c = ctx->cfg;
+  LaunchScope scope(ctx, MEDA_K_SELECT, as_stream(stream));
+  select_topk_kernel<<<c.n_kv_heads, kSelThreads, 0, as_stream(stream)>>>(
+      scores, ctx->ws.modality, budgets + (size_t)layer * 3, idx_conserved, idx_less, c.n_tokens, out_capacity,
+      ctx->ws.status);
+  return launch_status();
+}
+
+meda_status meda_merge_kv(meda_ctx* ctx, int32_t layer, const void* k, const void* v, const int32_t* budgets,
+                          const int32_t* idx_conserved, const int32_t* idx_less, void* k_out, void* v_out,
+                          int32_t* counts, int32_t* target, int32_t out_capacity, void* stream) {
+  if (!layer_ok(ctx, layer) || !k || !v || !budgets || !idx_conserved || !idx_less || !k_out || !v_out || !counts)
+    return MEDA_ERR_INVALID_ARG;
+  if (out_capacity < 1) return MEDA_ERR_WORKSPACE;
+  int32_t* tgt = target ? target : ctx->ws.target;
+  const int32_t* row = budgets + (size_t)layer * 3;
+  if (ctx->cfg.dtype == MEDA_F32)
+    return launch_merge<float>(ctx, k, v, row, idx_conserved, idx_less, k_out, v_out, counts, tgt, out_capacity,
+                               as_stream(stream));
+  return launch_merge<__nv_bfloat16>(ctx, k, v, row, idx_conserved, idx_less, k_out, v_out, counts, tgt, out_capacity,
+                                     as_stream(stream));
+}
+
+meda_status meda_compress_layer(meda_ctx* ctx, int32_t layer, const void* k, const void* v, const float* scores,
+                                const int32_t* budgets, void* k_out, void* v_out, int32_t* counts,
+                                int32_t* idx_conserved, int32_t out_capacity, void* stream) {
+  if (!layer_ok(ctx, layer) || !k || !v || !scores || !budgets || !k_out || !v_out || !counts || !idx_conserved)
+    return MEDA_ERR_INVALID_ARG;
+  meda_status r = meda_select_topk(ctx, layer, scores, budgets, idx_conserved, ctx->ws.idx_less, out_capacity, stream);
+  if (r != MEDA_OK) return r;
+  return meda_merge_kv(ctx, layer, k, v, budgets, idx_conserved, ctx->ws.idx_less, k_out, v_out, counts, nullptr,
+                       out_capacity, stream);
+}
+
+}  // extern "C"
+#pragma GCC visibility pop

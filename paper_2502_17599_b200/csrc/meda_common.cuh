@@ -1,0 +1,94 @@
+// Shared declarations of the CUDA implementation: context layout, device status word, small
+// device helpers.  Nothing here is used by (or shared with) the CPU oracle.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/meda.h"
+
+namespace meda {
+
+constexpr int kMaxWindow = 128;
+constexpr int kMaxLayers = 1024;
+constexpr int kStatsChunks = 32;      // key chunks of the generic normaliser sweep
+constexpr int kGenericKeyTile = 64;   // keys per tile in the generic phase-A kernels
+constexpr float kCosEps = 1e-8f;      // lower clamp of a key norm (Eq. 11 is silent on zero norms)
+
+struct Workspace {
+  uint8_t* modality = nullptr;        // [n] 0 = text, 1 = visual
+  int* status = nullptr;              // device status word (first error wins)
+  float* stats_partial = nullptr;     // [chunks][Hq][w][4]
+  float* ent_partial = nullptr;       // [ent_slots]
+  float* inv_norm = nullptr;          // [Hkv][n]  1 / max(|k_c|, eps) per conserved slot
+  int32_t* target = nullptr;          // [Hkv][n]  used when the caller passes no target array
+  int32_t* idx_less = nullptr;        // [Hkv][n]  used by meda_compress_layer
+  int64_t bytes = 0;
+};
+
+}  // namespace meda
+
+namespace meda {
+// Optional per-launch timing: pairs of events recorded around kernel launches.
+struct Profiler {
+  static constexpr int kPool = 16384;
+  bool enabled = false;
+  cudaEvent_t* begin = nullptr;   // [kPool]
+  cudaEvent_t* end = nullptr;     // [kPool]
+  int* klass = nullptr;           // [kPool]
+  int used = 0;
+};
+}  // namespace meda
+
+struct meda_ctx {
+  meda_config cfg;
+  meda::Profiler prof;
+  int64_t launches = 0;
+  int device = 0;
+  int sm_count = 0;
+  int group = 1;          // query heads per KV head
+  int n_visual = 0;
+  int ent_slots = 0;      // entries of ent_partial written by one entropy sweep
+  meda::Workspace ws;
+};
+
+namespace meda {
+
+template <typename T>
+__device__ __forceinline__ float to_f32(T x);
+template <>
+__device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T>
+__device__ __forceinline__ T from_f32(float x);
+template <>
+__device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// First error wins; later ones are dropped.
+__device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// (m, z) <- merge of two online-softmax states; an empty state is (-inf, 0).
+__device__ __forceinline__ void merge_mz(float& m, float& z, float m2, float z2) {
+  float mn = fmaxf(m, m2);
+  if (mn == -INFINITY) { m = mn; z = 0.f; return; }
+  z = z * __expf(m - mn) + z2 * __expf(m2 - mn);
+  m = mn;
+}
+
+}  // namespace meda

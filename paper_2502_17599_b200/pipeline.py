@@ -1,0 +1,86 @@
+"""The whole compression pass as a user calls it: phase A for every layer, the budget barrier,
+phase B for every layer.  Only sequencing and buffer plumbing live here; every step is a C-ABI
+call into libmeda.so (see binding.py) and nothing runs on the CPU in between."""
+from __future__ import annotations
+
+import torch
+
+from . import binding
+from .workloads import Workload
+
+
+class CompressionPass:
+    """Buffers and call sequence of one prompt's pass on one GPU.
+
+    Outputs are packed: layer l's compacted caches occupy rows [offset_l, offset_l + S_l) of
+    `k_out` / `v_out` ([n_kv_heads] x rows x head_dim each), with offset_l = l * row_capacity.
+    `row_capacity` bounds S_l per layer (n_tokens is always safe; a smaller value saves memory and
+    makes a layer whose budget exceeds it report MEDA_ERR_WORKSPACE)."""
+
+    def __init__(self, wl: Workload, row_capacity: int | None = None, device="cuda", **ctx_overrides):
+        self.wl = wl
+        self.device = device
+        self.ctx = binding.Context.for_workload(wl, **ctx_overrides)
+        n, hkv, hq, w, d, L = wl.n_tokens, wl.n_kv_heads, wl.n_q_heads, wl.window, wl.head_dim, wl.n_layers
+        self.cap = n if row_capacity is None else int(row_capacity)
+        f32, i32 = torch.float32, torch.int32
+        self.row_stats = torch.empty((hq, w, 4), dtype=f32, device=device)
+        self.scores = torch.empty((L, hkv, n), dtype=f32, device=device)
+        self.entropy = torch.zeros(L, dtype=f32, device=device)
+        self.budgets = torch.zeros((L, 3), dtype=i32, device=device)
+        self.k_out = torch.empty((L, hkv, self.cap, d), dtype=wl.torch_dtype, device=device)
+        self.v_out = torch.empty((L, hkv, self.cap, d), dtype=wl.torch_dtype, device=device)
+        self.counts = torch.empty((L, hkv, self.cap), dtype=i32, device=device)
+        self.idx_c = torch.empty((L, hkv, self.cap), dtype=i32, device=device)
+
+    def close(self):
+        self.ctx.close()
+
+    def run(self, q_layers, k_layers, v_layers, stream=None):
+        """Enqueues the whole pass on `stream` (default: torch's current stream).  Inputs are lists
+        of per-layer device tensors.  Results stay on the device in this object's buffers."""
+        L = self.wl.n_layers
+        c = self.ctx
+        for l in range(L):
+            c.window_scores(l, q_layers[l], k_layers[l], self.row_stats, self.scores[l], self.entropy, stream)
+        c.allocate_budgets(self.entropy, self.budgets, stream)
+        for l in range(L):
+            c.compress_layer(l, k_layers[l], v_layers[l], self.scores[l], self.budgets, self.k_out[l], self.v_out[l],
+                             self.counts[l], self.idx_c[l], self.cap, stream)
+
+    def run_from_host(self, q_host, k_host, v_host, staging, out_host):
+        """End-to-end variant: per-layer inputs in pinned HOST memory are copied to the device
+        staging buffers, the pass runs, and the budgets plus the compacted caches (only the S_l live
+        rows of each layer) are copied back to pinned host memory: out_host[name][l] has S_l rows per
+        head (see `alloc_host_outputs`).  Returns (h2d_bytes, d2h_bytes)."""
+        L = self.wl.n_layers
+        h2d = 0
+        for l in range(L):
+            for src, dst in ((q_host[l], staging["q"][l]), (k_host[l], staging["k"][l]), (v_host[l], staging["v"][l])):
+                dst.copy_(src, non_blocking=True)
+                h2d += src.numel() * src.element_size()
+        self.run(staging["q"], staging["k"], staging["v"])
+        out_host["budgets"].copy_(self.budgets, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the live row counts decide what comes back
+        d2h = self.budgets.numel() * 4
+        for l in range(L):
+            s = int(out_host["budgets"][l, 0])
+            for name, src in (("k", self.k_out), ("v", self.v_out), ("counts", self.counts), ("idx", self.idx_c)):
+                out_host[name][l].copy_(src[l][:, :s], non_blocking=True)
+                d2h += src[l][:, :s].numel() * src.element_size()
+        torch.cuda.current_stream().synchronize()
+        return h2d, d2h
+
+    def alloc_host_outputs(self):
+        """Pinned host buffers sized by the budgets of the last run (budgets are a deterministic
+        function of the inputs, so a repeated run of the same prompt fits them exactly)."""
+        b = self.budgets.cpu()
+        wl = self.wl
+        out = dict(budgets=torch.empty_like(b).pin_memory(), k=[], v=[], counts=[], idx=[])
+        for l in range(wl.n_layers):
+            s = int(b[l, 0])
+            out["k"].append(torch.empty((wl.n_kv_heads, s, wl.head_dim), dtype=wl.torch_dtype).pin_memory())
+            out["v"].append(torch.empty((wl.n_kv_heads, s, wl.head_dim), dtype=wl.torch_dtype).pin_memory())
+            out["counts"].append(torch.empty((wl.n_kv_heads, s), dtype=torch.int32).pin_memory())
+            out["idx"].append(torch.empty((wl.n_kv_heads, s), dtype=torch.int32).pin_memory())
+        return out

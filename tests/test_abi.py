@@ -1,0 +1,83 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU and exports every function that
+include/meda.h declares; host-side argument checks answer before any CUDA call."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2502_17599_b200 import build, binding
+    build.build()
+    return binding.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "meda.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(meda_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(lib):
+    from paper_2502_17599_b200 import binding
+    names = declared_functions()
+    assert len(names) >= 11
+    for name in names:
+        assert hasattr(lib, name), name
+        assert name in binding.EXPORTS, name
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_status_strings(lib):
+    from paper_2502_17599_b200 import binding
+    assert binding.status_string(0) == "ok"
+    seen = {binding.status_string(s) for s in range(-7, 1)}
+    assert len(seen) == 8
+
+
+def test_create_rejects_bad_arguments_before_touching_the_device(lib):
+    from paper_2502_17599_b200 import binding as B
+    good = dict(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_tokens=100, window=8, dtype="bf16",
+                global_budget=50, spans=((0, 10, 0), (10, 90, 1), (90, 100, 0)))
+
+    def status_of(**kw):
+        args = dict(good)
+        args.update(kw)
+        try:
+            B.Context(**args)
+        except B.MedaError as e:
+            return e.status
+        return 0
+
+    assert status_of(n_q_heads=3) == B.MEDA_ERR_SHAPE
+    assert status_of(head_dim=96) == B.MEDA_ERR_SHAPE
+    assert status_of(window=101) == B.MEDA_ERR_SHAPE
+    assert status_of(window=200, n_tokens=1000, spans=((0, 1000, 1),), global_budget=500) == B.MEDA_ERR_SHAPE
+    assert status_of(global_budget=3) == B.MEDA_ERR_BUDGET_INFEASIBLE
+    assert status_of(global_budget=201) == B.MEDA_ERR_BUDGET_INFEASIBLE
+    assert status_of(spans=((0, 10, 0), (11, 100, 1))) == B.MEDA_ERR_INVALID_ARG      # gap
+    assert status_of(spans=((0, 10, 0), (10, 90, 2), (90, 100, 0))) == B.MEDA_ERR_INVALID_ARG  # bad modality
+    assert status_of(spans=((0, 10, 0), (10, 90, 1))) == B.MEDA_ERR_INVALID_ARG        # does not cover
+    assert status_of(entropy_mode=2) == B.MEDA_ERR_INVALID_ARG
+    assert status_of(beta_recent=0, beta_important=0) == B.MEDA_ERR_INVALID_ARG
+
+
+def test_null_handles_are_rejected(lib):
+    assert lib.meda_poll_status(None, None) == -1
+    assert lib.meda_allocate_budgets(None, None, None, None) == -1
+    assert lib.meda_window_scores(None, 0, None, None, None, None, None, None) == -1
+    assert lib.meda_workspace_bytes(None) == 0
+    lib.meda_destroy(None)
+
+
+def test_product_path_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2502_17599_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "from oracle" not in text, f

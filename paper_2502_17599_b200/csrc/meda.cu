@@ -12,6 +12,7 @@
 #include "attn_generic.cuh"
 #include "meda_common.cuh"
 #include "merge_generic.cuh"
+#include "nearest_sm100.cuh"
 #include "select.cuh"
 
 using namespace meda;
@@ -47,6 +48,8 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.inv_norm);
   cudaFree(ws.target);
   cudaFree(ws.idx_less);
+  cudaFree(ws.kc);
+  cudaFree(ws.token_target);
   ws = Workspace();
 }
 
@@ -135,7 +138,68 @@ meda_status launch_sweep(meda_ctx* ctx, int32_t layer, const void* q_win, const 
   return launch_status();
 }
 
+// ---- TMA descriptors ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+void* resolve_encode_tiled() {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess)
+    return nullptr;
+  return fn;
+}
+
+// bf16 tensor [heads][rows][128] (row-major, dense) as a 3-D map with 64-column x box_rows boxes and
+// the 128-byte swizzle the UMMA operand descriptors expect.  Out-of-range rows read as zeros.
+bool make_rows_map(const meda_ctx* ctx, CUtensorMap* map, const void* base, int64_t rows, int64_t heads,
+                   int64_t head_stride_rows, uint32_t box_rows) {
+  cuuint64_t dims[3] = {(cuuint64_t)kFastDim, (cuuint64_t)rows, (cuuint64_t)heads};
+  cuuint64_t strides[2] = {(cuuint64_t)kFastDim * 2, (cuuint64_t)head_stride_rows * kFastDim * 2};
+  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint32_t elem[3] = {1, 1, 1};
+  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // ---- phase B launches ------------------------------------------------------------------------
+// bf16, head_dim 128: gather + tcgen05 similarity/arg-max + remap to the less-important order.
+meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* budget_row, const int32_t* idx_conserved,
+                                const int32_t* idx_less, int32_t* target, int32_t cap, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const int n = c.n_tokens;
+  if ((reinterpret_cast<uintptr_t>(k) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
+  CUtensorMap map_k, map_kc;
+  if (!make_rows_map(ctx, &map_k, k, n, c.n_kv_heads, n, 128) ||
+      !make_rows_map(ctx, &map_kc, ctx->ws.kc, ctx->kc_rows, c.n_kv_heads, ctx->kc_rows, kNnTileN))
+    return MEDA_ERR_CUDA;
+  const int max_slots = std::min(cap, n);
+  {
+    LaunchScope scope(ctx, MEDA_K_PREP, st);
+    gather_conserved_bf16_kernel<<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(k), idx_conserved, budget_row, ctx->ws.kc, ctx->ws.inv_norm, n, cap,
+        ctx->kc_rows, ctx->inv_stride);
+  }
+  {
+    const int items = ((n + kNnBlockM - 1) / kNnBlockM) * c.n_kv_heads;
+    LaunchScope scope(ctx, MEDA_K_NEAREST, st);
+    nearest_sm100_kernel<<<std::min(items, ctx->sm_count), kNnThreads, NnShared::alloc, st>>>(
+        map_k, map_kc, ctx->ws.inv_norm, budget_row, ctx->ws.token_target, n, c.n_kv_heads, cap, ctx->inv_stride,
+        ctx->ws.status);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_GROUP, st);
+    remap_targets_kernel<<<dim3((n + 255) / 256, c.n_kv_heads), 256, 0, st>>>(ctx->ws.token_target, idx_less,
+                                                                              budget_row, target, n, cap);
+  }
+  return launch_status();
+}
+
 template <typename T>
 meda_status launch_merge(meda_ctx* ctx, const void* k, const void* v, const int32_t* budget_row,
                          const int32_t* idx_conserved, const int32_t* idx_less, void* k_out, void* v_out,
@@ -144,16 +208,20 @@ meda_status launch_merge(meda_ctx* ctx, const void* k, const void* v, const int3
   const int n = c.n_tokens, d = c.head_dim;
   const int max_slots = std::min(cap, n);
   const int evict = c.merge_mode == 1;
-  if (!evict) {
+  if (!evict && ctx->fast) {
+    meda_status r = launch_nearest_fast(ctx, k, budget_row, idx_conserved, idx_less, target, cap, st);
+    if (r != MEDA_OK) return r;
+  } else if (!evict) {
     {
       LaunchScope scope(ctx, MEDA_K_PREP, st);
       conserved_inv_norm_kernel<T><<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
-          static_cast<const T*>(k), idx_conserved, budget_row, ctx->ws.inv_norm, n, d, cap);
+          static_cast<const T*>(k), idx_conserved, budget_row, ctx->ws.inv_norm, n, d, cap, ctx->inv_stride);
     }
     const int nn_smem = (kNnTile * (d + 1) + kNnTile * (kNnDk + 1)) * 4;
     LaunchScope scope(ctx, MEDA_K_NEAREST, st);
     nearest_generic_kernel<T><<<dim3((n + kNnTile - 1) / kNnTile, c.n_kv_heads), 256, nn_smem, st>>>(
-        static_cast<const T*>(k), idx_conserved, idx_less, budget_row, ctx->ws.inv_norm, target, n, d, cap);
+        static_cast<const T*>(k), idx_conserved, idx_less, budget_row, ctx->ws.inv_norm, target, n, d, cap,
+        ctx->inv_stride);
   }
   LaunchScope scope(ctx, MEDA_K_REDUCE, st);
   merge_scan_kernel<T><<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
@@ -232,7 +300,23 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   if (st == MEDA_OK) st = carve(&ws.status, 1, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.stats_partial, (int64_t)kStatsChunks * c.n_q_heads * c.window * 4, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
-  if (st == MEDA_OK) st = carve(&ws.inv_norm, hkv * n, &ws.bytes);
+  ctx->fast = c.dtype == MEDA_BF16 && c.head_dim == kFastDim;
+  ctx->kc_rows = (int)((n + 127) / 128 * 128);
+  ctx->inv_stride = ctx->kc_rows + 128;
+  if (st == MEDA_OK) st = carve(&ws.inv_norm, hkv * ctx->inv_stride, &ws.bytes);
+  if (ctx->fast) {
+    if (st == MEDA_OK) st = carve(&ws.kc, hkv * ctx->kc_rows * kFastDim, &ws.bytes);
+    if (st == MEDA_OK) st = carve(&ws.token_target, hkv * n, &ws.bytes);
+    if (st == MEDA_OK && cudaMemset(ws.kc, 0, (size_t)(hkv * ctx->kc_rows * kFastDim * 2)) != cudaSuccess) st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK && cudaMemset(ws.inv_norm, 0, (size_t)(hkv * ctx->inv_stride * 4)) != cudaSuccess) st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK) {
+      ctx->encode_tiled = resolve_encode_tiled();
+      if (!ctx->encode_tiled) st = MEDA_ERR_CUDA;
+    }
+    if (st == MEDA_OK && cudaFuncSetAttribute(nearest_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)NnShared::alloc) != cudaSuccess)
+      st = MEDA_ERR_CUDA;
+  }
   if (st == MEDA_OK) st = carve(&ws.target, hkv * n, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.idx_less, hkv * n, &ws.bytes);
   if (st == MEDA_OK && cudaMemcpy(ws.modality, modality.data(), (size_t)n, cudaMemcpyHostToDevice) != cudaSuccess)

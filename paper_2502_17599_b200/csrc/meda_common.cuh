@@ -21,7 +21,9 @@ struct Workspace {
   int* status = nullptr;              // device status word (first error wins)
   float* stats_partial = nullptr;     // [chunks][Hq][w][4]
   float* ent_partial = nullptr;       // [ent_slots]
-  float* inv_norm = nullptr;          // [Hkv][n]  1 / max(|k_c|, eps) per conserved slot
+  float* inv_norm = nullptr;          // [Hkv][inv_stride]  1 / max(|k_c|, eps) per conserved slot
+  __nv_bfloat16* kc = nullptr;        // [Hkv][kc_rows][128] gathered conserved keys (bf16, head_dim 128 only)
+  int32_t* token_target = nullptr;    // [Hkv][n] nearest slot of every token row (tensor-core path)
   int32_t* target = nullptr;          // [Hkv][n]  used when the caller passes no target array
   int32_t* idx_less = nullptr;        // [Hkv][n]  used by meda_compress_layer
   int64_t bytes = 0;
@@ -50,6 +52,10 @@ struct meda_ctx {
   int group = 1;          // query heads per KV head
   int n_visual = 0;
   int ent_slots = 0;      // entries of ent_partial written by one entropy sweep
+  int inv_stride = 0;     // floats per head in ws.inv_norm (padded so 128-wide slices can be read whole)
+  int kc_rows = 0;        // rows per head in ws.kc
+  bool fast = false;      // bf16 with head_dim 128: tensor-core kernels are used
+  void* encode_tiled = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
   meda::Workspace ws;
 };
 

@@ -11,7 +11,7 @@ namespace meda {
 template <typename T>
 __global__ void conserved_inv_norm_kernel(const T* __restrict__ k, const int32_t* __restrict__ idx_conserved,
                                           const int32_t* __restrict__ budget_row, float* __restrict__ inv_norm,
-                                          int n, int d, int cap) {
+                                          int n, int d, int cap, int inv_stride) {
   const int g = blockIdx.y;
   const int S = min(budget_row[0], cap);
   const int slot = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
@@ -23,7 +23,7 @@ __global__ void conserved_inv_norm_kernel(const T* __restrict__ k, const int32_t
   float ss = 0.f;
   for (int t = lane; t < d; t += 32) { float x = to_f32<T>(kr[t]); ss = fmaf(x, x, ss); }
   ss = warp_sum(ss);
-  if (lane == 0) inv_norm[(size_t)g * n + slot] = 1.f / fmaxf(sqrtf(ss), kCosEps);
+  if (lane == 0) inv_norm[(size_t)g * inv_stride + slot] = 1.f / fmaxf(sqrtf(ss), kCosEps);
 }
 
 // target[g][p] = argmax over slots s of k[less_p] . k[c_s] * inv_norm[s]  (the row's own norm is a
@@ -36,7 +36,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 nearest_generic_kernel(const T* __restrict__ k, const int32_t* __restrict__ idx_conserved,
                        const int32_t* __restrict__ idx_less, const int32_t* __restrict__ budget_row,
-                       const float* __restrict__ inv_norm, int32_t* __restrict__ target, int n, int d, int cap) {
+                       const float* __restrict__ inv_norm, int32_t* __restrict__ target, int n, int d, int cap,
+                       int inv_stride) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* a_s = reinterpret_cast<float*>(smem_raw);               // [64][d + 1]
   float* b_s = a_s + kNnTile * (d + 1);                          // [64][kNnDk + 1]
@@ -48,7 +49,7 @@ nearest_generic_kernel(const T* __restrict__ k, const int32_t* __restrict__ idx_
   const T* k_g = k + (size_t)g * n * d;
   const int32_t* less = idx_less + (size_t)g * n;
   const int32_t* cons = idx_conserved + (size_t)g * cap;
-  const float* inv = inv_norm + (size_t)g * n;
+  const float* inv = inv_norm + (size_t)g * inv_stride;
   const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
 
   for (int e = threadIdx.x; e < kNnTile * d; e += 256) {

@@ -1,0 +1,319 @@
+// Phase B, merge step 2 (Eq. 12): average every conserved row with the less-important rows
+// assigned to it, for keys and values, deterministically.
+//
+// The less-important rows are first grouped by target slot with a stable least-significant-digit
+// radix sort (9-bit digits; stability keeps the rows of a slot in ascending token order), so every
+// slot's members are contiguous and ordered.  Warps then walk fixed 128-row chunks of the sorted
+// list, summing in fp32 in list order; a slot whose members lie inside one chunk is finished on the
+// spot (own row first, then its members, one division, one rounding), pieces of slots that cross
+// chunk borders are parked as partial sums and added up in chunk order by a second small kernel.
+// No floating-point atomics anywhere: two runs give identical bits.
+#pragma once
+
+#include "meda_common.cuh"
+
+namespace meda {
+
+constexpr int kSortBits = 9;
+constexpr int kSortBins = 1 << kSortBits;
+constexpr int kSortChunk = 1024;      // elements ranked by one warp
+constexpr int kSortWarps = 8;
+constexpr int kSegChunk = 128;        // sorted rows walked by one warp
+constexpr int kSegWarps = 8;
+
+// ---- stable radix pass: histogram, scan, scatter ----------------------------------------------
+// table[g][bin][chunk] <- number of keys of warp-chunk `chunk` whose digit is `bin`.
+__global__ void __launch_bounds__(kSortWarps * 32)
+sort_hist_kernel(const int32_t* __restrict__ keys, const int32_t* __restrict__ budget_row, int32_t* __restrict__ table,
+                 int n, int cap, int shift, int n_chunks) {
+  __shared__ int cnt[kSortWarps][kSortBins];
+  const int g = blockIdx.y, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int chunk = blockIdx.x * kSortWarps + warp;
+  if (chunk >= n_chunks) return;
+  const int n_less = n - min(budget_row[0], cap);
+  for (int b = lane; b < kSortBins; b += 32) cnt[warp][b] = 0;
+  __syncwarp();
+  const int32_t* kg = keys + (size_t)g * n;
+  for (int r = 0; r < kSortChunk / 32; ++r) {
+    int q = chunk * kSortChunk + r * 32 + lane;
+    if (q < n_less) atomicAdd(&cnt[warp][(kg[q] >> shift) & (kSortBins - 1)], 1);
+  }
+  __syncwarp();
+  int32_t* tg = table + (size_t)g * kSortBins * n_chunks;
+  for (int b = lane; b < kSortBins; b += 32) tg[(size_t)b * n_chunks + chunk] = cnt[warp][b];
+}
+
+// In-place exclusive prefix sum of each head's table in (bin, chunk) order.  One block per head.
+__global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ table, int len) {
+  __shared__ int warp_sums[32];
+  int32_t* t = table + (size_t)blockIdx.x * len;
+  const int per = (len + 1023) / 1024;
+  const int begin = min((int)threadIdx.x * per, len), end = min(begin + per, len);
+  int sum = 0;
+  for (int e = begin; e < end; ++e) sum += t[e];
+  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+  int incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums[lane], wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += y;
+    }
+    warp_sums[lane] = wi - w;
+  }
+  __syncthreads();
+  int run = warp_sums[warp] + incl - sum;
+  for (int e = begin; e < end; ++e) {
+    int x = t[e];
+    t[e] = run;
+    run += x;
+  }
+}
+
+// Stable scatter of (key, row) pairs by the digit at `shift`, using the scanned table.
+__global__ void __launch_bounds__(kSortWarps * 32)
+sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restrict__ rows_in,
+                    const int32_t* __restrict__ budget_row, const int32_t* __restrict__ table,
+                    int32_t* __restrict__ keys_out, int32_t* __restrict__ rows_out, int n, int cap, int shift,
+                    int n_chunks) {
+  __shared__ int cnt[kSortWarps][kSortBins];
+  const int g = blockIdx.y, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int chunk = blockIdx.x * kSortWarps + warp;
+  if (chunk >= n_chunks) return;
+  const int n_less = n - min(budget_row[0], cap);
+  if (chunk * kSortChunk >= n_less) return;
+  const int32_t* tg = table + (size_t)g * kSortBins * n_chunks;
+  for (int b = lane; b < kSortBins; b += 32) cnt[warp][b] = tg[(size_t)b * n_chunks + chunk];
+  __syncwarp();
+  const int32_t* kg = keys_in + (size_t)g * n;
+  const int32_t* rg = rows_in + (size_t)g * n;
+  int32_t* ko = keys_out + (size_t)g * n;
+  int32_t* ro = rows_out + (size_t)g * n;
+  const unsigned int lt = (1u << lane) - 1u;
+  for (int r = 0; r < kSortChunk / 32; ++r) {
+    const int q = chunk * kSortChunk + r * 32 + lane;
+    const bool valid = q < n_less;
+    const int key = valid ? kg[q] : 0;
+    const int row = valid ? rg[q] : 0;
+    const int digit = (key >> shift) & (kSortBins - 1);
+    const unsigned int peers = __match_any_sync(0xffffffffu, valid ? digit : kSortBins + lane);
+    const int leader = __ffs(peers) - 1;
+    int base = 0;
+    if (valid && lane == leader) {
+      base = cnt[warp][digit];
+      cnt[warp][digit] = base + __popc(peers);
+    }
+    base = __shfl_sync(0xffffffffu, base, leader);
+    if (valid) {
+      const int pos = min(base + __popc(peers & lt), n - 1);
+      ko[pos] = key;
+      ro[pos] = row;
+    }
+    __syncwarp();
+  }
+}
+
+// ---- segmented average ---------------------------------------------------------------------------
+// Layout of the parked partial sums: piece `which` (0 = head: the slot started in an earlier chunk,
+// 1 = tail: it started here and continues) of chunk c of head g holds 2*D floats (keys then values).
+template <int D>
+__device__ __forceinline__ float* carry_ptr(float* carry, int g, int chunk, int which, int n_chunks) {
+  return carry + (((size_t)g * n_chunks + chunk) * 2 + which) * (2 * D);
+}
+
+template <typename T, int E>
+__device__ __forceinline__ void load_row(const T* p, int lane, float (&x)[E]);
+
+template <>
+__device__ __forceinline__ void load_row<__nv_bfloat16, 2>(const __nv_bfloat16* p, int lane, float (&x)[2]) {
+  float2 a = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(p)[lane]);
+  x[0] = a.x; x[1] = a.y;
+}
+template <>
+__device__ __forceinline__ void load_row<__nv_bfloat16, 4>(const __nv_bfloat16* p, int lane, float (&x)[4]) {
+  uint2 u = reinterpret_cast<const uint2*>(p)[lane];
+  float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&u.x));
+  float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&u.y));
+  x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+}
+template <>
+__device__ __forceinline__ void load_row<__nv_bfloat16, 8>(const __nv_bfloat16* p, int lane, float (&x)[8]) {
+  uint4 u = reinterpret_cast<const uint4*>(p)[lane];
+  float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&u.x));
+  float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&u.y));
+  float2 c = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&u.z));
+  float2 d = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&u.w));
+  x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y; x[4] = c.x; x[5] = c.y; x[6] = d.x; x[7] = d.y;
+}
+template <>
+__device__ __forceinline__ void load_row<float, 2>(const float* p, int lane, float (&x)[2]) {
+  float2 a = reinterpret_cast<const float2*>(p)[lane];
+  x[0] = a.x; x[1] = a.y;
+}
+template <>
+__device__ __forceinline__ void load_row<float, 4>(const float* p, int lane, float (&x)[4]) {
+  float4 a = reinterpret_cast<const float4*>(p)[lane];
+  x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+}
+template <>
+__device__ __forceinline__ void load_row<float, 8>(const float* p, int lane, float (&x)[8]) {
+  float4 a = reinterpret_cast<const float4*>(p)[2 * lane], b = reinterpret_cast<const float4*>(p)[2 * lane + 1];
+  x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+
+// Lane `lane` owns elements [lane * E, lane * E + E) of a row.
+template <typename T, int E>
+__device__ __forceinline__ void store_row(T* p, int lane, const float (&x)[E], float count) {
+#pragma unroll
+  for (int e = 0; e < E; ++e) p[lane * E + e] = from_f32<T>(x[e] / count);
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kSegWarps * 32)
+seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ keys,
+                  const int32_t* __restrict__ rows, const int32_t* __restrict__ idx_conserved,
+                  const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,
+                  int32_t* __restrict__ counts, int32_t* __restrict__ seg_start, int32_t* __restrict__ seg_end,
+                  float* __restrict__ carry, int32_t* __restrict__ carry_cnt, int n, int cap, int n_chunks) {
+  constexpr int E = D / 32;
+  const int g = blockIdx.y, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int chunk = blockIdx.x * kSegWarps + warp;
+  const int S = min(budget_row[0], cap);
+  const int n_less = n - S;
+  const int q0 = chunk * kSegChunk;
+  if (q0 >= n_less) return;
+  const int q1 = min(q0 + kSegChunk, n_less);
+  const int32_t* kg = keys + (size_t)g * n;
+  const int32_t* rg = rows + (size_t)g * n;
+  const T* k_g = k + (size_t)g * n * D;
+  const T* v_g = v + (size_t)g * n * D;
+  const int32_t* cons = idx_conserved + (size_t)g * cap;
+  int32_t* st = seg_start + (size_t)g * n;
+  int32_t* en = seg_end + (size_t)g * n;
+
+  float ak[E], av[E];
+  int members = 0;
+  int cur = min(max(kg[q0], 0), S - 1);
+  bool started_here = (q0 == 0) || (kg[q0 - 1] != kg[q0]);
+
+  auto begin_segment = [&](int slot, bool fresh, int q) {
+    members = 0;
+    if (fresh) {
+      const int own = min(max(cons[slot], 0), n - 1);
+      load_row<T, E>(k_g + (size_t)own * D, lane, ak);
+      load_row<T, E>(v_g + (size_t)own * D, lane, av);
+      if (lane == 0) st[slot] = q;
+    } else {
+#pragma unroll
+      for (int e = 0; e < E; ++e) { ak[e] = 0.f; av[e] = 0.f; }
+    }
+  };
+  auto end_piece = [&](int slot, bool fresh, bool ended, int q_end) {
+    if (ended && lane == 0) en[slot] = q_end;
+    if (fresh && ended) {
+      const float c = (float)(members + 1);
+      store_row<T, E>(k_out + ((size_t)g * cap + slot) * D, lane, ak, c);
+      store_row<T, E>(v_out + ((size_t)g * cap + slot) * D, lane, av, c);
+      if (lane == 0) counts[(size_t)g * cap + slot] = members + 1;
+    } else {
+      const int which = fresh ? 1 : 0;
+      float* cp = carry_ptr<D>(carry, g, chunk, which, n_chunks);
+#pragma unroll
+      for (int e = 0; e < E; ++e) { cp[lane * E + e] = ak[e]; cp[D + lane * E + e] = av[e]; }
+      if (lane == 0) carry_cnt[((size_t)g * n_chunks + chunk) * 2 + which] = members;
+    }
+  };
+
+  begin_segment(cur, started_here, q0);
+  constexpr int kBatch = 8;
+  for (int qb = q0; qb < q1; qb += kBatch) {
+    float xk[kBatch][E], xv[kBatch][E];
+    int key[kBatch];
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const int q = min(qb + b, q1 - 1);
+      key[b] = min(max(kg[q], 0), S - 1);
+      const int row = min(max(rg[q], 0), n - 1);
+      load_row<T, E>(k_g + (size_t)row * D, lane, xk[b]);
+      load_row<T, E>(v_g + (size_t)row * D, lane, xv[b]);
+    }
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      if (qb + b < q1) {
+        if (key[b] != cur) {
+          end_piece(cur, started_here, true, qb + b);
+          cur = key[b];
+          started_here = true;
+          begin_segment(cur, true, qb + b);
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) { ak[e] += xk[b][e]; av[e] += xv[b][e]; }
+        ++members;
+      }
+    }
+  }
+  const bool ended = (q1 == n_less) || (min(max(kg[q1], 0), S - 1) != cur);
+  end_piece(cur, started_here, ended, q1);
+}
+
+// One warp per conserved slot: slots without members are copied, slots whose members span several
+// chunks get their parked pieces added in chunk order; everything else was finished by the walker.
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ idx_conserved,
+                    const int32_t* __restrict__ budget_row, const int32_t* __restrict__ seg_start,
+                    const int32_t* __restrict__ seg_end, const float* __restrict__ carry,
+                    const int32_t* __restrict__ carry_cnt, T* __restrict__ k_out, T* __restrict__ v_out,
+                    int32_t* __restrict__ counts, int n, int cap, int n_chunks, int evict) {
+  constexpr int E = D / 32;
+  const int g = blockIdx.y, lane = threadIdx.x % 32;
+  const int S = min(budget_row[0], cap);
+  const int slot = blockIdx.x * 8 + threadIdx.x / 32;
+  if (slot >= S) return;
+  const int start = evict ? 0 : seg_start[(size_t)g * n + slot];
+  const int end = evict ? 0 : seg_end[(size_t)g * n + slot];
+  float ak[E], av[E];
+  int members = 0;
+  if (end <= start) {
+    const int own = min(max(idx_conserved[(size_t)g * cap + slot], 0), n - 1);
+    load_row<T, E>(k + ((size_t)g * n + own) * D, lane, ak);
+    load_row<T, E>(v + ((size_t)g * n + own) * D, lane, av);
+  } else {
+    const int c0 = start / kSegChunk, c1 = (end - 1) / kSegChunk;
+    if (c0 == c1) return;
+    float* base = const_cast<float*>(carry);
+    const float* p = carry_ptr<D>(base, g, c0, 1, n_chunks);
+#pragma unroll
+    for (int e = 0; e < E; ++e) { ak[e] = p[lane * E + e]; av[e] = p[D + lane * E + e]; }
+    members = carry_cnt[((size_t)g * n_chunks + c0) * 2 + 1];
+    for (int c = c0 + 1; c <= c1; ++c) {
+      p = carry_ptr<D>(base, g, c, 0, n_chunks);
+#pragma unroll
+      for (int e = 0; e < E; ++e) { ak[e] += p[lane * E + e]; av[e] += p[D + lane * E + e]; }
+      members += carry_cnt[((size_t)g * n_chunks + c) * 2];
+    }
+  }
+  const float c = (float)(members + 1);
+  store_row<T, E>(k_out + ((size_t)g * cap + slot) * D, lane, ak, c);
+  store_row<T, E>(v_out + ((size_t)g * cap + slot) * D, lane, av, c);
+  if (lane == 0) counts[(size_t)g * cap + slot] = members + 1;
+}
+
+// Clears the per-slot segment bounds of one layer (slots without members must read as empty).
+__global__ void clear_segments_kernel(int32_t* __restrict__ seg_start, int32_t* __restrict__ seg_end,
+                                      const int32_t* __restrict__ budget_row, int n, int cap) {
+  const int g = blockIdx.y;
+  const int S = min(budget_row[0], cap);
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s < S) { seg_start[(size_t)g * n + s] = 0; seg_end[(size_t)g * n + s] = 0; }
+}
+
+}  // namespace meda

@@ -11,6 +11,7 @@
 #include "allocate.cuh"
 #include "attn_generic.cuh"
 #include "meda_common.cuh"
+#include "group_reduce.cuh"
 #include "merge_generic.cuh"
 #include "nearest_sm100.cuh"
 #include "select.cuh"
@@ -50,6 +51,12 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.idx_less);
   cudaFree(ws.kc);
   cudaFree(ws.token_target);
+  for (int i = 0; i < 2; ++i) { cudaFree(ws.sort_keys[i]); cudaFree(ws.sort_rows[i]); }
+  cudaFree(ws.sort_table);
+  cudaFree(ws.seg_start);
+  cudaFree(ws.seg_end);
+  cudaFree(ws.carry);
+  cudaFree(ws.carry_cnt);
   ws = Workspace();
 }
 
@@ -200,6 +207,75 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
   return launch_status();
 }
 
+// Grouping sort + segmented average (Eq. 12) for any dtype / head_dim.
+template <typename T, int D>
+void launch_seg_kernels(meda_ctx* ctx, const void* k, const void* v, const int32_t* budget_row,
+                        const int32_t* idx_conserved, const int32_t* keys, const int32_t* rows, void* k_out,
+                        void* v_out, int32_t* counts, int32_t cap, int evict, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const int n = c.n_tokens;
+  const int max_slots = std::min(cap, n);
+  if (!evict) {
+    LaunchScope scope(ctx, MEDA_K_REDUCE, st);
+    seg_reduce_kernel<T, D><<<dim3((ctx->seg_chunks + kSegWarps - 1) / kSegWarps, c.n_kv_heads), kSegWarps * 32, 0, st>>>(
+        static_cast<const T*>(k), static_cast<const T*>(v), keys, rows, idx_conserved, budget_row,
+        static_cast<T*>(k_out), static_cast<T*>(v_out), counts, ctx->ws.seg_start, ctx->ws.seg_end, ctx->ws.carry,
+        ctx->ws.carry_cnt, n, cap, ctx->seg_chunks);
+  }
+  LaunchScope scope(ctx, MEDA_K_REDUCE, st);
+  seg_finalize_kernel<T, D><<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
+      static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, budget_row, ctx->ws.seg_start,
+      ctx->ws.seg_end, ctx->ws.carry, ctx->ws.carry_cnt, static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n,
+      cap, ctx->seg_chunks, evict);
+}
+
+template <typename T>
+meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, const int32_t* budget_row,
+                                const int32_t* idx_conserved, const int32_t* idx_less, const int32_t* target,
+                                void* k_out, void* v_out, int32_t* counts, int32_t cap, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const int n = c.n_tokens;
+  const int evict = c.merge_mode == 1;
+  const int max_slots = std::min(cap, n);
+  const int32_t* keys = target;
+  const int32_t* rows = idx_less;
+  if (!evict) {
+    {
+      LaunchScope scope(ctx, MEDA_K_GROUP, st);
+      clear_segments_kernel<<<dim3((max_slots + 255) / 256, c.n_kv_heads), 256, 0, st>>>(ctx->ws.seg_start,
+                                                                                       ctx->ws.seg_end, budget_row, n, cap);
+    }
+    const dim3 grid((ctx->sort_chunks + kSortWarps - 1) / kSortWarps, c.n_kv_heads);
+    for (int pass = 0; pass < ctx->sort_passes; ++pass) {
+      int32_t* ko = ctx->ws.sort_keys[pass & 1];
+      int32_t* ro = ctx->ws.sort_rows[pass & 1];
+      const int shift = pass * kSortBits;
+      {
+        LaunchScope scope(ctx, MEDA_K_GROUP, st);
+        sort_hist_kernel<<<grid, kSortWarps * 32, 0, st>>>(keys, budget_row, ctx->ws.sort_table, n, cap, shift,
+                                                           ctx->sort_chunks);
+      }
+      {
+        LaunchScope scope(ctx, MEDA_K_GROUP, st);
+        sort_scan_kernel<<<c.n_kv_heads, 1024, 0, st>>>(ctx->ws.sort_table, kSortBins * ctx->sort_chunks);
+      }
+      {
+        LaunchScope scope(ctx, MEDA_K_GROUP, st);
+        sort_scatter_kernel<<<grid, kSortWarps * 32, 0, st>>>(keys, rows, budget_row, ctx->ws.sort_table, ko, ro, n,
+                                                              cap, shift, ctx->sort_chunks);
+      }
+      keys = ko;
+      rows = ro;
+    }
+  }
+  switch (c.head_dim) {
+    case 64: launch_seg_kernels<T, 64>(ctx, k, v, budget_row, idx_conserved, keys, rows, k_out, v_out, counts, cap, evict, st); break;
+    case 128: launch_seg_kernels<T, 128>(ctx, k, v, budget_row, idx_conserved, keys, rows, k_out, v_out, counts, cap, evict, st); break;
+    default: launch_seg_kernels<T, 256>(ctx, k, v, budget_row, idx_conserved, keys, rows, k_out, v_out, counts, cap, evict, st); break;
+  }
+  return launch_status();
+}
+
 template <typename T>
 meda_status launch_merge(meda_ctx* ctx, const void* k, const void* v, const int32_t* budget_row,
                          const int32_t* idx_conserved, const int32_t* idx_less, void* k_out, void* v_out,
@@ -223,11 +299,7 @@ meda_status launch_merge(meda_ctx* ctx, const void* k, const void* v, const int3
         static_cast<const T*>(k), idx_conserved, idx_less, budget_row, ctx->ws.inv_norm, target, n, d, cap,
         ctx->inv_stride);
   }
-  LaunchScope scope(ctx, MEDA_K_REDUCE, st);
-  merge_scan_kernel<T><<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
-      static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, idx_less, target, budget_row,
-      static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n, d, cap, evict);
-  return launch_status();
+  return launch_group_reduce<T>(ctx, k, v, budget_row, idx_conserved, idx_less, target, k_out, v_out, counts, cap, st);
 }
 
 }  // namespace
@@ -300,6 +372,18 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   if (st == MEDA_OK) st = carve(&ws.status, 1, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.stats_partial, (int64_t)kStatsChunks * c.n_q_heads * c.window * 4, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
+  ctx->sort_chunks = (int)((n + kSortChunk - 1) / kSortChunk);
+  ctx->seg_chunks = (int)((n + kSegChunk - 1) / kSegChunk);
+  ctx->sort_passes = n <= kSortBins ? 1 : (n <= (int64_t)kSortBins * kSortBins ? 2 : 3);
+  for (int i = 0; i < 2; ++i) {
+    if (st == MEDA_OK) st = carve(&ws.sort_keys[i], hkv * n, &ws.bytes);
+    if (st == MEDA_OK) st = carve(&ws.sort_rows[i], hkv * n, &ws.bytes);
+  }
+  if (st == MEDA_OK) st = carve(&ws.sort_table, hkv * kSortBins * ctx->sort_chunks, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.seg_start, hkv * n, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.seg_end, hkv * n, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.carry, hkv * ctx->seg_chunks * 2 * 2 * c.head_dim, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.carry_cnt, hkv * ctx->seg_chunks * 2, &ws.bytes);
   ctx->fast = c.dtype == MEDA_BF16 && c.head_dim == kFastDim;
   ctx->kc_rows = (int)((n + 127) / 128 * 128);
   ctx->inv_stride = ctx->kc_rows + 128;

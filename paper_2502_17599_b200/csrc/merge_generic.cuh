@@ -1,6 +1,6 @@
 // Phase B, merging (Eq. 11-12), dtype-generic CUDA-core kernels: inverse norms of the conserved
-// keys, nearest conserved key of every less-important key (cosine similarity, first maximum), and
-// the average merge itself.  These are the fp32 path and the bring-up path for bf16.
+// keys and nearest conserved key of every less-important key (cosine similarity, first maximum).
+// These are the fp32 path and the path for head dimensions the tensor-core kernel does not cover.
 #pragma once
 
 #include "meda_common.cuh"
@@ -120,67 +120,6 @@ nearest_generic_kernel(const T* __restrict__ k, const int32_t* __restrict__ idx_
     int p = r0 + ty * 4 + r;
     if (tx == 0 && p < n_less) target[(size_t)g * n + p] = s;
   }
-}
-
-// Average merge (Eq. 12) by one warp per conserved slot: walks the less-important list in
-// ascending order and adds the rows assigned to its slot (fp32, fixed order), then divides by
-// the member count and rounds once.  Work is O(S * n_less) reads of the target array.
-template <typename T>
-__global__ void __launch_bounds__(256)
-merge_scan_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ idx_conserved,
-                  const int32_t* __restrict__ idx_less, const int32_t* __restrict__ target,
-                  const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,
-                  int32_t* __restrict__ counts, int n, int d, int cap, int evict) {
-  const int g = blockIdx.y;
-  const int S = min(budget_row[0], cap);
-  const int slot = blockIdx.x * 8 + threadIdx.x / 32;
-  if (slot >= S) return;
-  const int lane = threadIdx.x % 32;
-  const int n_less = n - S;
-  const T* k_g = k + (size_t)g * n * d;
-  const T* v_g = v + (size_t)g * n * d;
-  const int nd = d / 32;   // <= 8
-  float ak[8], av[8];
-  int own = min(max(idx_conserved[(size_t)g * cap + slot], 0), n - 1);
-#pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    if (c < nd) {
-      ak[c] = to_f32<T>(k_g[(size_t)own * d + c * 32 + lane]);
-      av[c] = to_f32<T>(v_g[(size_t)own * d + c * 32 + lane]);
-    }
-  }
-  int count = 1;
-  if (!evict) {
-    const int32_t* tg = target + (size_t)g * n;
-    const int32_t* less = idx_less + (size_t)g * n;
-    for (int p0 = 0; p0 < n_less; p0 += 32) {
-      int p = p0 + lane;
-      bool mine = p < n_less && tg[p] == slot;
-      unsigned int ballot = __ballot_sync(0xffffffffu, mine);
-      while (ballot) {
-        int b = __ffs(ballot) - 1;
-        ballot &= ballot - 1;
-        int row = min(max(less[p0 + b], 0), n - 1);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          if (c < nd) {
-            ak[c] += to_f32<T>(k_g[(size_t)row * d + c * 32 + lane]);
-            av[c] += to_f32<T>(v_g[(size_t)row * d + c * 32 + lane]);
-          }
-        }
-        ++count;
-      }
-    }
-  }
-  const float cf = (float)count;
-#pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    if (c < nd) {
-      k_out[((size_t)g * cap + slot) * d + c * 32 + lane] = from_f32<T>(ak[c] / cf);
-      v_out[((size_t)g * cap + slot) * d + c * 32 + lane] = from_f32<T>(av[c] / cf);
-    }
-  }
-  if (lane == 0) counts[(size_t)g * cap + slot] = count;
 }
 
 }  // namespace meda

@@ -1,0 +1,297 @@
+// Phase A for bf16 / head_dim 128 on the tensor cores (Eq. 4-6 and Eq. 8 with the query rows
+// restricted to the observation window).  Two policies of the streaming UMMA pipeline:
+//
+//  StatsPolicy  (sweep 1)  resident block = the window rows of one KV group (rows = (head, window
+//               row)), streamed tiles = 128 keys each; every epilogue thread owns one query row and
+//               keeps online softmax normalisers (max, sum of exp2) separately over visual and text
+//               keys.  One exp2 per logit.
+//  SweepPolicy  (sweep 2)  resident block = 256 keys of one KV head (rows = keys), streamed tiles =
+//               the group's window rows, 128 columns each; every epilogue thread owns one key: it sums
+//               the normalised probabilities of its key over all columns (the accumulated score,
+//               Eq. 8) and keeps the head-averaged text-to-vision attention of its key for every
+//               window row across the KV heads, from which the entropy partial follows (Eq. 5).
+//               One exp2 per logit serves both the full and the visual-only softmax.
+//
+// Logits are kept in base-2 units: t = (q.k) * scale * log2(e).
+#pragma once
+
+#include "umma_stream.cuh"
+
+namespace meda {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sweep 1: normalisers
+// ---------------------------------------------------------------------------------------------
+struct StatsPolicy {
+  struct Params {
+    const uint8_t* modality;     // padded to a multiple of 128 with the value 2 (= no key)
+    float* partial;              // [chunks][Hq][w][4]
+    int n, hq, group, w, cols;   // cols = group * w query rows per KV group
+    int row_blocks;              // ceil(cols / 256)
+    int chunks, tiles_per_chunk, tiles_total;
+    float sc2;                   // scale * log2(e)
+  };
+  static constexpr int kABuffers = 1;
+  static constexpr int kBStages = 4;
+  static constexpr uint32_t kExtraBytes = kUsEpilogueWarps * 128;     // one modality slice per epilogue warp
+
+  __device__ static bool active(const Params&) { return true; }
+  __device__ static bool get_item(const Params& p, int it, StreamItem& o) {
+    const int idx = blockIdx.x + it * gridDim.x;
+    const int per_group = p.row_blocks * p.chunks;
+    const int n_groups = p.hq / p.group;
+    if (idx >= per_group * n_groups) return false;
+    const int g = idx / per_group, rb = (idx / p.chunks) % p.row_blocks, kc = idx % p.chunks;
+    o.a_row = g * p.cols + rb * 256;
+    o.a_head = 0;
+    o.b_row = kc * p.tiles_per_chunk * 128;
+    o.b_head = g;
+    o.n_tiles = min(p.tiles_per_chunk, p.tiles_total - kc * p.tiles_per_chunk);
+    o.last_n = 128;
+    o.m_tiles = (p.cols - rb * 256 > 128) ? 2 : 1;
+    o.u0 = g * 65536 + rb;        // group and row block
+    o.u1 = kc;
+    return o.n_tiles > 0;
+  }
+
+  struct Epilogue {
+    uint8_t* mod_t;
+    int lane, row_in_block;
+    float mv, zv, mt, zt;        // running (max, sum) in base-2 logit units, visual and text keys
+    __device__ void init(const Params&, unsigned char* extra, int ewarp, int lane_) {
+      mod_t = extra + ewarp * 128;
+      lane = lane_;
+      row_in_block = (ewarp / 4) * 128 + ((ewarp + 2) % 4) * 32 + lane_;
+    }
+    __device__ void item_begin(const Params&, const StreamItem&) {
+      mv = mt = -INFINITY;
+      zv = zt = 0.f;
+    }
+    __device__ __forceinline__ static void absorb(float& m, float& z, float t) {
+      if (t > m) { z = z * fast_exp2(m - t) + 1.f; m = t; }
+      else z += fast_exp2(t - m);
+    }
+    __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
+      const int rb = it.u0 & 65535;
+      const int r = rb * 256 + row_in_block;            // query row inside the KV group
+      const bool valid = r < p.cols;
+      const int i = r % p.w;
+      const int last_visible = p.n - p.w + i;           // causal: keys j <= last_visible
+      const int c0 = it.b_row + tile * 128;
+      __syncwarp();
+      reinterpret_cast<uint32_t*>(mod_t)[lane] = __ldg(reinterpret_cast<const uint32_t*>(p.modality + c0) + lane);
+      __syncwarp();
+      if (!__any_sync(0xffffffffu, valid)) return;
+#pragma unroll 1
+      for (int chunk = 0; chunk < 4; ++chunk) {
+        float v[32];
+        __syncwarp();
+        sm100::tmem_ld_32x32(taddr + chunk * 32u, v);
+        if (valid) {
+        const int j0 = c0 + chunk * 32;
+        const uint4 ma = reinterpret_cast<const uint4*>(mod_t + chunk * 32)[0];
+        const uint4 mb = reinterpret_cast<const uint4*>(mod_t + chunk * 32)[1];
+        const uint32_t all_or = ma.x | ma.y | ma.z | ma.w | mb.x | mb.y | mb.z | mb.w;
+        const uint32_t all_and = ma.x & ma.y & ma.z & ma.w & mb.x & mb.y & mb.z & mb.w;
+        const bool uniform_text = all_or == 0u;
+        const bool uniform_visual = all_and == 0x01010101u && all_or == 0x01010101u;
+        if ((uniform_text || uniform_visual) && j0 + 31 <= last_visible) {
+          float cm = v[0];
+#pragma unroll
+          for (int x = 1; x < 32; ++x) cm = fmaxf(cm, v[x]);
+          float& m = uniform_visual ? mv : mt;
+          float& z = uniform_visual ? zv : zt;
+          const float m_new = fmaxf(m, cm * p.sc2);
+          float acc = 0.f;
+#pragma unroll
+          for (int x = 0; x < 32; ++x) acc += fast_exp2(fmaf(v[x], p.sc2, -m_new));
+          z = z * fast_exp2(m - m_new) + acc;
+          m = m_new;
+        } else {
+#pragma unroll
+          for (int x = 0; x < 32; ++x) {
+            const int md = mod_t[chunk * 32 + x];
+            if (md < 2 && j0 + x <= last_visible) {
+              if (md == MEDA_VISUAL) absorb(mv, zv, v[x] * p.sc2);
+              else absorb(mt, zt, v[x] * p.sc2);
+            }
+          }
+        }
+        }
+      }
+    }
+    __device__ void item_end(const Params& p, const StreamItem& it) {
+      const int g = it.u0 >> 16, rb = it.u0 & 65535;
+      const int r = rb * 256 + row_in_block;
+      if (r >= p.cols) return;
+      const int h = g * p.group + r / p.w, i = r % p.w;
+      // all keys = visual and text together
+      const float m_all = fmaxf(mv, mt);
+      float z_all = 0.f;
+      if (m_all > -INFINITY) z_all = zv * fast_exp2(mv - m_all) + zt * fast_exp2(mt - m_all);
+      float4 out;
+      out.x = m_all * kLn2;
+      out.y = z_all;
+      out.z = mv * kLn2;
+      out.w = zv;
+      reinterpret_cast<float4*>(p.partial)[((size_t)it.u1 * p.hq + h) * p.w + i] = out;
+    }
+  };
+};
+
+// ---------------------------------------------------------------------------------------------
+// Per-column constants of sweep 2, from the normalisers.
+//   vis[c]  = (m_vis * log2e, exp(m_vis - m_all) / z_all, 1 / (z_vis * Hq), -ln z_vis)   for visual keys
+//   text[c] = (m_all * log2e, 1 / z_all)                                                  for text keys
+// so that one e = exp2(t - ref) gives the full-softmax probability e * [1] and, for a visual key,
+// the head-averaged visual-softmax probability e * [2].
+// ---------------------------------------------------------------------------------------------
+__global__ void sweep_coef_kernel(const float* __restrict__ row_stats, float4* __restrict__ vis,
+                                  float2* __restrict__ text, int rows, float inv_hq) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= rows) return;
+  const float4 s = reinterpret_cast<const float4*>(row_stats)[c];
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (s.w > 0.f) {
+    a.x = s.z * kLog2e;
+    a.y = expf(s.z - s.x) / s.y;
+    a.z = inv_hq / s.w;
+    a.w = -logf(s.w);
+  }
+  vis[c] = a;
+  text[c] = make_float2(s.x * kLog2e, 1.f / s.y);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sweep 2: scores and entropy.  W = window (32 or 64).
+// ---------------------------------------------------------------------------------------------
+template <int W>
+struct SweepPolicy {
+  struct Params {
+    const uint8_t* modality;     // padded as above
+    const float4* vis;           // [Hq * w]
+    const float2* text;          // [Hq * w]
+    float* scores;               // [Hkv][n] or null
+    float* ent_partial;          // [blocks * 8] or null
+    int n, hkv, cols;            // cols = group * W columns per KV head
+    int n_blocks;                // ceil(n / 256)
+    int entropy_mode;
+    float sc2;
+  };
+  static constexpr int kABuffers = 2;
+  static constexpr int kBStages = 2;
+  static constexpr uint32_t kExtraBytes = 0;
+
+  __device__ static bool active(const Params&) { return true; }
+  // Each block takes whole 256-key blocks and walks all KV heads of a block back to back, so that
+  // the head-averaged attention of its keys is complete inside one thread.
+  __device__ static bool get_item(const Params& p, int it, StreamItem& o) {
+    const int blk = blockIdx.x + (it / p.hkv) * gridDim.x;
+    if (blk >= p.n_blocks) return false;
+    const int g = it % p.hkv;
+    o.a_row = blk * 256;
+    o.a_head = g;
+    o.b_row = g * p.cols;
+    o.b_head = 0;
+    o.n_tiles = (p.cols + 127) / 128;
+    o.last_n = p.cols - (o.n_tiles - 1) * 128;      // cols is a multiple of 32
+    o.m_tiles = (p.n - o.a_row > 128) ? 2 : 1;
+    o.u0 = g;
+    o.u1 = blk;
+    return true;
+  }
+
+  struct Epilogue {
+    int lane, ewarp, row_in_block;
+    float abar[W];               // head-averaged visual-softmax attention of this key, per window row
+    float plogp;                 // entropy_mode 1 accumulator
+    float score;
+    __device__ void init(const Params&, unsigned char*, int ewarp_, int lane_) {
+      lane = lane_;
+      ewarp = ewarp_;
+      row_in_block = (ewarp_ / 4) * 128 + ((ewarp_ + 2) % 4) * 32 + lane_;
+#pragma unroll
+      for (int x = 0; x < W; ++x) abar[x] = 0.f;
+      plogp = 0.f;
+    }
+    __device__ void item_begin(const Params&, const StreamItem&) { score = 0.f; }
+
+    template <int OFF>
+    __device__ __forceinline__ void chunk_visual(const Params& p, const float (&v)[32], int col0, int first_row) {
+#pragma unroll
+      for (int x = 0; x < 32; ++x) {
+        const float4 c = __ldg(p.vis + col0 + x);
+        const float t = fmaf(v[x], p.sc2, -c.x);
+        float e = fast_exp2(t);
+        if (OFF + x < first_row) e = 0.f;
+        score = fmaf(e, c.y, score);
+        const float pv = e * c.z;
+        if (p.entropy_mode == 0) abar[OFF + x] += pv;
+        else plogp = fmaf(pv, fmaf(t, kLn2, c.w), plogp);
+      }
+    }
+    __device__ __forceinline__ void chunk_text(const Params& p, const float (&v)[32], int col0, int row0, int first_row) {
+#pragma unroll
+      for (int x = 0; x < 32; ++x) {
+        const float2 c = __ldg(p.text + col0 + x);
+        float e = fast_exp2(fmaf(v[x], p.sc2, -c.x));
+        if (row0 + x < first_row) e = 0.f;
+        score = fmaf(e, c.y, score);
+      }
+    }
+    __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
+      const int j = it.a_row + row_in_block;               // this thread's key
+      const bool valid = j < p.n;
+      const int md = p.modality[j];                        // the padded map covers j up to the block end
+      const int first_row = j - (p.n - W);                 // causal: window rows i >= first_row see key j
+      const int n_chunks = (tile == it.n_tiles - 1 ? it.last_n : 128) / 32;
+#pragma unroll 1
+      for (int chunk = 0; chunk < n_chunks; ++chunk) {
+        float v[32];
+        __syncwarp();
+        sm100::tmem_ld_32x32(taddr + chunk * 32u, v);
+        if (valid) {
+          const int local = tile * 128 + chunk * 32;          // column inside the KV group: head * W + row
+          const int col0 = it.b_row + local;
+          const int row0 = local % W;
+          if (md == MEDA_VISUAL) {
+            if (W == 32 || row0 == 0) chunk_visual<0>(p, v, col0, first_row);
+            else chunk_visual<(W > 32 ? 32 : 0)>(p, v, col0, first_row);
+          } else {
+            chunk_text(p, v, col0, row0, first_row);
+          }
+        }
+      }
+    }
+    __device__ void item_end(const Params& p, const StreamItem& it) {
+      const int j = it.a_row + row_in_block;
+      if (p.scores && j < p.n) p.scores[(size_t)it.u0 * p.n + j] = score;
+      if (it.u0 == p.hkv - 1) {
+        // all heads of this key block are in: entropy partial of this warp's 32 keys
+        float acc = plogp;
+        if (p.entropy_mode == 0) {
+#pragma unroll
+          for (int x = 0; x < W; ++x) {
+            const float a = abar[x];
+            if (a > 0.f) acc = fmaf(a, __logf(a), acc);
+            abar[x] = 0.f;
+          }
+        }
+        plogp = 0.f;
+        acc = warp_sum(acc);
+        if (p.ent_partial && lane == 0) p.ent_partial[(size_t)it.u1 * kUsEpilogueWarps + ewarp] = acc;
+      }
+    }
+  };
+};
+
+}  // namespace meda

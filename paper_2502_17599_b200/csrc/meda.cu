@@ -10,6 +10,7 @@
 
 #include "allocate.cuh"
 #include "attn_generic.cuh"
+#include "attn_sm100.cuh"
 #include "meda_common.cuh"
 #include "group_reduce.cuh"
 #include "merge_generic.cuh"
@@ -51,6 +52,8 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.idx_less);
   cudaFree(ws.kc);
   cudaFree(ws.token_target);
+  cudaFree(ws.coef_vis);
+  cudaFree(ws.coef_text);
   for (int i = 0; i < 2; ++i) { cudaFree(ws.sort_keys[i]); cudaFree(ws.sort_rows[i]); }
   cudaFree(ws.sort_table);
   cudaFree(ws.seg_start);
@@ -104,6 +107,35 @@ void profiler_release(Profiler& p) {
 
 bool layer_ok(const meda_ctx* ctx, int32_t layer) { return ctx && layer >= 0 && layer < ctx->cfg.n_layers; }
 
+// ---- TMA descriptors ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+void* resolve_encode_tiled() {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess)
+    return nullptr;
+  return fn;
+}
+
+// bf16 tensor [heads][rows][128] (row-major, dense) as a 3-D map with 64-column x box_rows boxes and
+// the 128-byte swizzle the UMMA operand descriptors expect.  Out-of-range rows read as zeros.
+bool make_rows_map(const meda_ctx* ctx, CUtensorMap* map, const void* base, int64_t rows, int64_t heads,
+                   int64_t head_stride_rows, uint32_t box_rows) {
+  cuuint64_t dims[3] = {(cuuint64_t)kFastDim, (cuuint64_t)rows, (cuuint64_t)heads};
+  cuuint64_t strides[2] = {(cuuint64_t)kFastDim * 2, (cuuint64_t)head_stride_rows * kFastDim * 2};
+  cuuint32_t box[3] = {64, box_rows, 1};
+  cuuint32_t elem[3] = {1, 1, 1};
+  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // ---- phase A launches ------------------------------------------------------------------------
 template <typename T>
 meda_status launch_stats(meda_ctx* ctx, const void* q_win, const void* k, float* row_stats, cudaStream_t st) {
@@ -145,33 +177,80 @@ meda_status launch_sweep(meda_ctx* ctx, int32_t layer, const void* q_win, const 
   return launch_status();
 }
 
-// ---- TMA descriptors ---------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-void* resolve_encode_tiled() {
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-      q != cudaDriverEntryPointSuccess)
-    return nullptr;
-  return fn;
+// bf16, head_dim 128, window 32 or 64: both sweeps on the tensor cores.
+meda_status launch_stats_fast(meda_ctx* ctx, const void* q_win, const void* k, float* row_stats, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  if (((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(q_win)) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
+  CUtensorMap map_q, map_k;
+  if (!make_rows_map(ctx, &map_q, q_win, (int64_t)c.n_q_heads * c.window, 1, (int64_t)c.n_q_heads * c.window, 128) ||
+      !make_rows_map(ctx, &map_k, k, c.n_tokens, c.n_kv_heads, c.n_tokens, 128))
+    return MEDA_ERR_CUDA;
+  StatsPolicy::Params prm;
+  prm.modality = ctx->ws.modality;
+  prm.partial = ctx->ws.stats_partial;
+  prm.n = c.n_tokens; prm.hq = c.n_q_heads; prm.group = ctx->group; prm.w = c.window;
+  prm.cols = ctx->group * c.window;
+  prm.row_blocks = (prm.cols + 255) / 256;
+  prm.chunks = ctx->stats_chunks;
+  prm.tiles_per_chunk = ctx->stats_tiles_per_chunk;
+  prm.tiles_total = (c.n_tokens + 127) / 128;
+  prm.sc2 = kLog2e / sqrtf((float)c.head_dim);
+  const int items = c.n_kv_heads * prm.row_blocks * prm.chunks;
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS, st);
+    umma_stream_kernel<StatsPolicy><<<std::min(items, ctx->sm_count), kUsThreads, StreamShared<StatsPolicy>::alloc, st>>>(
+        map_q, map_k, prm, ctx->ws.status);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
+    stats_combine_kernel<<<c.n_q_heads, kMaxWindow, 0, st>>>(ctx->ws.stats_partial, row_stats, prm.chunks, c.n_q_heads, c.window);
+  }
+  return launch_status();
 }
 
-// bf16 tensor [heads][rows][128] (row-major, dense) as a 3-D map with 64-column x box_rows boxes and
-// the 128-byte swizzle the UMMA operand descriptors expect.  Out-of-range rows read as zeros.
-bool make_rows_map(const meda_ctx* ctx, CUtensorMap* map, const void* base, int64_t rows, int64_t heads,
-                   int64_t head_stride_rows, uint32_t box_rows) {
-  cuuint64_t dims[3] = {(cuuint64_t)kFastDim, (cuuint64_t)rows, (cuuint64_t)heads};
-  cuuint64_t strides[2] = {(cuuint64_t)kFastDim * 2, (cuuint64_t)head_stride_rows * kFastDim * 2};
-  cuuint32_t box[3] = {64, box_rows, 1};
-  cuuint32_t elem[3] = {1, 1, 1};
-  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
-      map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
-      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+template <int W>
+void launch_sweep_policy(meda_ctx* ctx, const CUtensorMap& map_k, const CUtensorMap& map_q, float* scores,
+                         bool want_entropy, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  typename SweepPolicy<W>::Params prm;
+  prm.modality = ctx->ws.modality;
+  prm.vis = ctx->ws.coef_vis;
+  prm.text = ctx->ws.coef_text;
+  prm.scores = scores;
+  prm.ent_partial = want_entropy ? ctx->ws.ent_partial : nullptr;
+  prm.n = c.n_tokens; prm.hkv = c.n_kv_heads; prm.cols = ctx->group * c.window;
+  prm.n_blocks = (c.n_tokens + 255) / 256;
+  prm.entropy_mode = c.entropy_mode;
+  prm.sc2 = kLog2e / sqrtf((float)c.head_dim);
+  umma_stream_kernel<SweepPolicy<W>><<<std::min(prm.n_blocks, ctx->sm_count), kUsThreads, StreamShared<SweepPolicy<W>>::alloc, st>>>(
+      map_k, map_q, prm, ctx->ws.status);
+}
+
+meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
+                              float* scores, float* entropy, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  if (((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(q_win)) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
+  CUtensorMap map_q, map_k;
+  if (!make_rows_map(ctx, &map_q, q_win, (int64_t)c.n_q_heads * c.window, 1, (int64_t)c.n_q_heads * c.window, 128) ||
+      !make_rows_map(ctx, &map_k, k, c.n_tokens, c.n_kv_heads, c.n_tokens, 128))
+    return MEDA_ERR_CUDA;
+  const int rows = c.n_q_heads * c.window;
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
+    sweep_coef_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_stats, ctx->ws.coef_vis, ctx->ws.coef_text, rows,
+                                                          1.0f / (float)c.n_q_heads);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_SWEEP, st);
+    if (c.window == 32) launch_sweep_policy<32>(ctx, map_k, map_q, scores, entropy != nullptr, st);
+    else launch_sweep_policy<64>(ctx, map_k, map_q, scores, entropy != nullptr, st);
+  }
+  if (entropy) {
+    LaunchScope scope(ctx, MEDA_K_ENTROPY_FINAL, st);
+    entropy_finalize_kernel<<<1, 256, 0, st>>>(ctx->ws.ent_partial, ((c.n_tokens + 255) / 256) * kUsEpilogueWarps,
+                                               row_stats, c.window, entropy + layer);
+  }
+  return launch_status();
 }
 
 // ---- phase B launches ------------------------------------------------------------------------
@@ -183,7 +262,7 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
   if ((reinterpret_cast<uintptr_t>(k) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
   CUtensorMap map_k, map_kc;
   if (!make_rows_map(ctx, &map_k, k, n, c.n_kv_heads, n, 128) ||
-      !make_rows_map(ctx, &map_kc, ctx->ws.kc, ctx->kc_rows, c.n_kv_heads, ctx->kc_rows, kNnTileN))
+      !make_rows_map(ctx, &map_kc, ctx->ws.kc, ctx->kc_rows, c.n_kv_heads, ctx->kc_rows, 128))
     return MEDA_ERR_CUDA;
   const int max_slots = std::min(cap, n);
   {
@@ -193,11 +272,11 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
         ctx->kc_rows, ctx->inv_stride);
   }
   {
-    const int items = ((n + kNnBlockM - 1) / kNnBlockM) * c.n_kv_heads;
+    const int items = ((n + 255) / 256) * c.n_kv_heads;
+    NearestPolicy::Params prm{ctx->ws.inv_norm, budget_row, ctx->ws.token_target, n, c.n_kv_heads, cap, ctx->inv_stride};
     LaunchScope scope(ctx, MEDA_K_NEAREST, st);
-    nearest_sm100_kernel<<<std::min(items, ctx->sm_count), kNnThreads, NnShared::alloc, st>>>(
-        map_k, map_kc, ctx->ws.inv_norm, budget_row, ctx->ws.token_target, n, c.n_kv_heads, cap, ctx->inv_stride,
-        ctx->ws.status);
+    umma_stream_kernel<NearestPolicy><<<std::min(items, ctx->sm_count), kUsThreads, StreamShared<NearestPolicy>::alloc, st>>>(
+        map_k, map_kc, prm, ctx->ws.status);
   }
   {
     LaunchScope scope(ctx, MEDA_K_GROUP, st);
@@ -363,14 +442,38 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     delete ctx;
     return MEDA_ERR_CUDA;
   }
-  ctx->ent_slots = generic_tiles(c.n_tokens);
+  ctx->fast = c.dtype == MEDA_BF16 && c.head_dim == kFastDim;
+  ctx->fast_attn = ctx->fast && (c.window == 32 || c.window == 64);
+  ctx->ent_slots = std::max(generic_tiles(c.n_tokens), ((c.n_tokens + 255) / 256) * kUsEpilogueWarps);
+  {
+    // key chunks of the tensor-core normaliser sweep: about two items per SM
+    const int tiles = (c.n_tokens + 127) / 128;
+    const int row_blocks = (ctx->group * c.window + 255) / 256;
+    int want = std::max(1, (2 * ctx->sm_count) / std::max(1, c.n_kv_heads * row_blocks));
+    want = std::min(want, tiles);
+    ctx->stats_tiles_per_chunk = (tiles + want - 1) / want;
+    ctx->stats_chunks = (tiles + ctx->stats_tiles_per_chunk - 1) / ctx->stats_tiles_per_chunk;
+  }
 
   Workspace& ws = ctx->ws;
   const int64_t n = c.n_tokens, hkv = c.n_kv_heads;
   meda_status st = MEDA_OK;
-  if (st == MEDA_OK) st = carve(&ws.modality, n, &ws.bytes);
+  const int64_t mod_bytes = (n + 255) / 256 * 256 + 128;
+  if (st == MEDA_OK) st = carve(&ws.modality, mod_bytes, &ws.bytes);
+  if (st == MEDA_OK && cudaMemset(ws.modality, 2, (size_t)mod_bytes) != cudaSuccess) st = MEDA_ERR_CUDA;
   if (st == MEDA_OK) st = carve(&ws.status, 1, &ws.bytes);
-  if (st == MEDA_OK) st = carve(&ws.stats_partial, (int64_t)kStatsChunks * c.n_q_heads * c.window * 4, &ws.bytes);
+  if (st == MEDA_OK)
+    st = carve(&ws.stats_partial, (int64_t)std::max(kStatsChunks, ctx->stats_chunks) * c.n_q_heads * c.window * 4, &ws.bytes);
+  if (ctx->fast_attn) {
+    if (st == MEDA_OK) st = carve(&ws.coef_vis, (int64_t)c.n_q_heads * c.window, &ws.bytes);
+    if (st == MEDA_OK) st = carve(&ws.coef_text, (int64_t)c.n_q_heads * c.window, &ws.bytes);
+    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<StatsPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)StreamShared<StatsPolicy>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<SweepPolicy<32>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)StreamShared<SweepPolicy<32>>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<SweepPolicy<64>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)StreamShared<SweepPolicy<64>>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
+  }
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
   ctx->sort_chunks = (int)((n + kSortChunk - 1) / kSortChunk);
   ctx->seg_chunks = (int)((n + kSegChunk - 1) / kSegChunk);
@@ -384,7 +487,6 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   if (st == MEDA_OK) st = carve(&ws.seg_end, hkv * n, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.carry, hkv * ctx->seg_chunks * 2 * 2 * c.head_dim, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.carry_cnt, hkv * ctx->seg_chunks * 2, &ws.bytes);
-  ctx->fast = c.dtype == MEDA_BF16 && c.head_dim == kFastDim;
   ctx->kc_rows = (int)((n + 127) / 128 * 128);
   ctx->inv_stride = ctx->kc_rows + 128;
   if (st == MEDA_OK) st = carve(&ws.inv_norm, hkv * ctx->inv_stride, &ws.bytes);
@@ -397,8 +499,8 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
       ctx->encode_tiled = resolve_encode_tiled();
       if (!ctx->encode_tiled) st = MEDA_ERR_CUDA;
     }
-    if (st == MEDA_OK && cudaFuncSetAttribute(nearest_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)NnShared::alloc) != cudaSuccess)
+    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<NearestPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)StreamShared<NearestPolicy>::alloc) != cudaSuccess)
       st = MEDA_ERR_CUDA;
   }
   if (st == MEDA_OK) st = carve(&ws.target, hkv * n, &ws.bytes);
@@ -496,7 +598,10 @@ meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, 
   if (!layer_ok(ctx, layer) || !q_win || !k || !row_stats || !scores) return MEDA_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
   meda_status r;
-  if (ctx->cfg.dtype == MEDA_F32) {
+  if (ctx->fast_attn) {
+    r = launch_stats_fast(ctx, q_win, k, row_stats, st);
+    if (r == MEDA_OK) r = launch_sweep_fast(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+  } else if (ctx->cfg.dtype == MEDA_F32) {
     r = launch_stats<float>(ctx, q_win, k, row_stats, st);
     if (r == MEDA_OK) r = launch_sweep<float>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
   } else {
@@ -512,6 +617,7 @@ meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, 
   if (!layer_ok(ctx, layer) || !q_win || !k || !row_stats || !entropy) return MEDA_ERR_INVALID_ARG;
   if (q_vis || q_vis_pos || n_vis_rows != 0) return MEDA_ERR_UNSUPPORTED;
   cudaStream_t st = as_stream(stream);
+  if (ctx->fast_attn) return launch_sweep_fast(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
   if (ctx->cfg.dtype == MEDA_F32) return launch_sweep<float>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
   return launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
 }

@@ -17,7 +17,9 @@ constexpr int kGenericKeyTile = 64;   // keys per tile in the generic phase-A ke
 constexpr float kCosEps = 1e-8f;      // lower clamp of a key norm (Eq. 11 is silent on zero norms)
 
 struct Workspace {
-  uint8_t* modality = nullptr;        // [n] 0 = text, 1 = visual
+  uint8_t* modality = nullptr;        // [n padded to a multiple of 256, + 128] 0 = text, 1 = visual, 2 = padding
+  float4* coef_vis = nullptr;         // [Hq * w] per-column constants of the tensor-core scores sweep
+  float2* coef_text = nullptr;        // [Hq * w]
   int* status = nullptr;              // device status word (first error wins)
   float* stats_partial = nullptr;     // [chunks][Hq][w][4]
   float* ent_partial = nullptr;       // [ent_slots]
@@ -65,6 +67,9 @@ struct meda_ctx {
   int seg_chunks = 0;     // warp-chunks per head in the segmented average
   int sort_passes = 1;    // 9-bit digit passes needed to order slots < n_tokens
   bool fast = false;      // bf16 with head_dim 128: tensor-core kernels are used
+  bool fast_attn = false; // ... and window 32 or 64: phase A runs on the tensor cores too
+  int stats_chunks = 0;   // key chunks of the tensor-core normaliser sweep
+  int stats_tiles_per_chunk = 0;
   void* encode_tiled = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
   meda::Workspace ws;
 };

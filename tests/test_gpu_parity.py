@@ -25,6 +25,10 @@ def small_cases():
         W.small_variant(),                                   # bf16, GQA 3:1, ragged n = 661
         W.small_variant("small_mha_d64", n_q_heads=4, n_kv_heads=4, head_dim=64, window=17, seed=2),
         W.small_variant("small_f32_gqa", dtype="f32", n_q_heads=4, n_kv_heads=2, head_dim=128, seed=3),
+        # shapes that take the tensor-core phase-A kernels (bf16, d=128, window 32 or 64)
+        W.small_variant("tc_w32", window=32, seed=4),
+        W.small_variant("tc_w64_wide", window=64, n_q_heads=10, n_kv_heads=2, seed=5),   # 320 query rows per KV group
+        W.WORKLOADS["long_video_19k"].with_(name="long_video_19k_2l", n_layers=2),
     ]
 
 

@@ -509,11 +509,10 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     st = MEDA_ERR_CUDA;
   if (st == MEDA_OK && cudaMemset(ws.status, 0, sizeof(int)) != cudaSuccess) st = MEDA_ERR_CUDA;
   if (st == MEDA_OK) {
-    const int stats_smem = attn_generic_smem(c.window, c.head_dim, false).total;
-    const int sweep_smem = attn_generic_smem(c.window, c.head_dim, true).total;
-    const int nn_smem = (kNnTile * (c.head_dim + 1) + kNnTile * (kNnDk + 1)) * 4;
-    st = c.dtype == MEDA_F32 ? set_generic_attrs<float>(stats_smem, sweep_smem, nn_smem)
-                             : set_generic_attrs<__nv_bfloat16>(stats_smem, sweep_smem, nn_smem);
+    // The limit is a property of the kernel, not of the context: always raise it to the ceiling so
+    // that contexts of different shapes can coexist.
+    st = c.dtype == MEDA_F32 ? set_generic_attrs<float>(kMaxDynSmem, kMaxDynSmem, kMaxDynSmem)
+                             : set_generic_attrs<__nv_bfloat16>(kMaxDynSmem, kMaxDynSmem, kMaxDynSmem);
   }
   if (st != MEDA_OK) {
     free_workspace(ws);

@@ -273,3 +273,18 @@ def test_end_to_end_with_teacher_forcing(wl):
                              host[l][1][g], host[l][2][g], cons, less, tgt, wl.dtype)
     print(f"{wl.name}: tolerated selection swaps {swaps}, tolerated arg-max near-ties {ties}")
     ctx.close()
+
+
+def test_contexts_of_different_shapes_coexist():
+    """A context created later with a smaller shape must not shrink what an earlier one may launch."""
+    big = W.small_variant("coexist_big", dtype="f32", n_q_heads=2, n_kv_heads=2, window=96, seed=6)
+    small = W.small_variant("coexist_small", dtype="f32", n_q_heads=2, n_kv_heads=2, window=8, seed=6)
+    ctx_big = make_ctx(big)
+    ctx_small = make_ctx(small)
+    buf = P.GpuBuffers(big)
+    (q, k, v), (qh, kh, vh) = P.layer_inputs(big, 0, "cuda")
+    ctx_big.window_scores(0, q, k, buf.row_stats, buf.scores, buf.entropy)
+    ctx_big.check()
+    P.assert_scores_close(P.np64(buf.scores), O.window_scores(qh, kh))
+    ctx_small.close()
+    ctx_big.close()

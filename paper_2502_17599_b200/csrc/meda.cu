@@ -65,12 +65,24 @@ void free_workspace(Workspace& ws) {
 
 int generic_tiles(int n) { return (n + kGenericKeyTile - 1) / kGenericKeyTile; }
 
-template <typename T>
-meda_status set_generic_attrs(int stats_smem, int sweep_smem, int nn_smem) {
-  MEDA_CUDA_TRY(cudaFuncSetAttribute(stats_partial_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, stats_smem));
-  MEDA_CUDA_TRY(cudaFuncSetAttribute(scores_entropy_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, sweep_smem));
-  MEDA_CUDA_TRY(cudaFuncSetAttribute(nearest_generic_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, nn_smem));
+// Raises a kernel's dynamic shared memory limit to the most the SM offers next to the kernel's
+// static shared memory.  The limit belongs to the kernel, not to a context, so it is never set
+// to one context's need: contexts of different shapes coexist.
+template <typename K>
+meda_status raise_dyn_smem(K kernel) {
+  cudaFuncAttributes a;
+  MEDA_CUDA_TRY(cudaFuncGetAttributes(&a, kernel));
+  MEDA_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kMaxDynSmem - (int)a.sharedSizeBytes));
   return MEDA_OK;
+}
+
+template <typename T>
+meda_status set_generic_attrs() {
+  meda_status r = raise_dyn_smem(stats_partial_kernel<T>);
+  if (r == MEDA_OK) r = raise_dyn_smem(scores_entropy_kernel<T>);
+  if (r == MEDA_OK) r = raise_dyn_smem(nearest_generic_kernel<T>);
+  return r;
 }
 
 // Brackets one kernel launch with profiling events (when enabled) and counts it.
@@ -511,8 +523,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   if (st == MEDA_OK) {
     // The limit is a property of the kernel, not of the context: always raise it to the ceiling so
     // that contexts of different shapes can coexist.
-    st = c.dtype == MEDA_F32 ? set_generic_attrs<float>(kMaxDynSmem, kMaxDynSmem, kMaxDynSmem)
-                             : set_generic_attrs<__nv_bfloat16>(kMaxDynSmem, kMaxDynSmem, kMaxDynSmem);
+    st = c.dtype == MEDA_F32 ? set_generic_attrs<float>() : set_generic_attrs<__nv_bfloat16>();
   }
   if (st != MEDA_OK) {
     free_workspace(ws);

@@ -158,6 +158,45 @@ meda_status meda_compress_layer(meda_ctx* ctx, int32_t layer, const void* k, con
                                 const int32_t* budgets, void* k_out, void* v_out, int32_t* counts,
                                 int32_t* idx_conserved, int32_t out_capacity, void* stream);
 
+/* ---- entry point that allocates nothing (the paper has no counterpart) ---------------------- */
+
+/* Largest n_q_heads * window the entry point below accepts, and the size of the scratch array
+ * it uses: MEDA_STATIC_STATS_CHUNKS partial results of 4 floats for each of those rows (2 MiB). */
+enum { MEDA_STATIC_STATS_MAX_ROWS = 4096, MEDA_STATIC_STATS_CHUNKS = 32 };
+
+/* Softmax normalisers of the window rows (the row_stats array of meda_window_scores, same
+ * layout and meaning) for callers that cannot allocate device memory.  Every other entry point
+ * needs a context, and meda_create calls cudaMalloc.  A serving process that handed the whole of
+ * device memory to its own pool at start-up has none left for cudaMalloc to hand out; a caller in
+ * the middle of a latency-critical section cannot afford the device-wide synchronisation that
+ * cudaMalloc and cudaFree imply; both can still call this function.  It takes no context, calls
+ * no allocating routine, and keeps its only scratch memory, the per-key-chunk partial
+ * normalisers, in a fixed 2 MiB array inside the library's device image: every GPU that loads
+ * the library holds those 2 MiB until the process exits, whether this function is called or not.
+ *
+ *   q_win    device, `dtype`, [n_q_heads][window][head_dim]
+ *   k        device, `dtype`, [n_kv_heads][n_tokens][head_dim]
+ *   modality device, uint8 [n_tokens]: MEDA_TEXT or MEDA_VISUAL per token (the caller's own map;
+ *            there is no context to build it from a span table)
+ *   row_stats device output, fp32 [n_q_heads][window][4], fully overwritten
+ *
+ * Limits: n_q_heads * window <= MEDA_STATIC_STATS_MAX_ROWS, window <= 128, head_dim in {64, 128,
+ * 256}, n_q_heads a multiple of n_kv_heads; anything else returns MEDA_ERR_SHAPE (or
+ * MEDA_ERR_INVALID_ARG for NULL pointers or an unknown dtype) before any CUDA call.
+ * It always runs the CUDA-core kernels, so for bf16 / head_dim 128 / window 32 or 64 its numbers
+ * agree with meda_window_scores' to rounding (2e-5 on the log-normaliser), not bit for bit.
+ *
+ * The first call on each device looks up the scratch array's device address and raises the
+ * kernel's shared-memory limit, with that device current; make that first call before any stream
+ * capture begins.  Later calls on the device only launch.  The array is shared by every call in
+ * the process: each call overwrites all the entries it later reads, so nothing needs clearing
+ * and the last call's contents are harmless, but two calls whose kernels overlap on the same GPU
+ * (different streams, or different host threads) race on it and give wrong results; serialise
+ * them. */
+meda_status meda_row_stats_static(const void* q_win, const void* k, const uint8_t* modality,
+                                  int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t n_tokens,
+                                  int32_t window, int32_t dtype, float* row_stats, void* stream);
+
 /* ---- measurement helpers (no counterpart in the paper) ------------------------------------ */
 
 /* Kernel classes the library reports times for. */

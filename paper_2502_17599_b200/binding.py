@@ -67,6 +67,7 @@ EXPORTS = {
     "meda_window_scores": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
     "meda_layer_entropy": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 5 +
                            [ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]),
+    "meda_row_stats_static": (ctypes.c_int, [ctypes.c_void_p] * 3 + [ctypes.c_int32] * 6 + [ctypes.c_void_p] * 2),
     "meda_allocate_budgets": (ctypes.c_int, [ctypes.c_void_p] * 4),
     "meda_select_topk": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
                          [ctypes.c_int32, ctypes.c_void_p]),
@@ -118,6 +119,23 @@ def _stream(stream):
 def _check(status: int, where: str):
     if status != MEDA_OK:
         raise MedaError(status, where)
+
+
+STATIC_STATS_MAX_ROWS = 4096
+
+
+def row_stats_static(q_win, k, modality, row_stats, stream=None):
+    """meda_row_stats_static: the window rows' softmax normalisers without a context and without
+    any device allocation, for callers that cannot call cudaMalloc (all of device memory already
+    belongs to their own pool, or they are inside a section that must not synchronise the device).
+    Shapes are read from the tensors: q_win [Hq, w, d], k [Hkv, n, d], modality uint8 [n],
+    row_stats fp32 [Hq, w, 4].  Calls that overlap on one GPU race on the library's fixed scratch
+    array; the first call on a device should come before any stream capture."""
+    hq, w, d = q_win.shape
+    hkv, n, _ = k.shape
+    dtype = MEDA_F32 if q_win.dtype == torch.float32 else MEDA_BF16
+    _check(load_library().meda_row_stats_static(_ptr(q_win), _ptr(k), _ptr(modality), hq, hkv, d, n, w, dtype,
+                                                _ptr(row_stats), _stream(stream)), "meda_row_stats_static")
 
 
 class Context:

@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -395,8 +396,85 @@ meda_status launch_merge(meda_ctx* ctx, const void* k, const void* v, const int3
 
 }  // namespace
 
+// ---- scratch and set-up of meda_row_stats_static -----------------------------------------------
+// The partial normalisers of the entry point that must not allocate: [chunks][rows][4] floats at the
+// largest size it accepts.  This name is only a device address inside device code; host code must
+// ask the runtime for the address (static_stats_scratch below) and never pass the name to a kernel.
+static __device__ __align__(256) float g_static_stats_partial[(size_t)MEDA_STATIC_STATS_CHUNKS *
+                                                             MEDA_STATIC_STATS_MAX_ROWS * 4];
+static_assert(MEDA_STATIC_STATS_CHUNKS == meda::kStatsChunks, "the static scratch is sized for the generic sweep");
+
+namespace {
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticStatsDevice {
+  float* partial = nullptr;   // device address of g_static_stats_partial on this device
+  bool ready = false;
+};
+StaticStatsDevice g_static_stats_devices[kStaticMaxDevices];
+std::mutex g_static_stats_mutex;
+
+// Once per device, with that device current: the array's device address and the kernels' shared
+// memory limit.  Neither call allocates.  Returns the address through *partial.
+meda_status static_stats_scratch(float** partial) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return MEDA_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_stats_mutex);
+  StaticStatsDevice& d = g_static_stats_devices[dev];
+  if (!d.ready) {
+    float* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_stats_partial) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return MEDA_ERR_CUDA;
+    }
+    if (raise_dyn_smem(stats_partial_kernel<float>) != MEDA_OK || raise_dyn_smem(stats_partial_kernel<__nv_bfloat16>) != MEDA_OK)
+      return MEDA_ERR_CUDA;
+    d.partial = ptr;
+    d.ready = true;
+  }
+  *partial = d.partial;
+  return MEDA_OK;
+}
+
+}  // namespace
+
 #pragma GCC visibility push(default)
 extern "C" {
+
+meda_status meda_row_stats_static(const void* q_win, const void* k, const uint8_t* modality, int32_t n_q_heads,
+                                  int32_t n_kv_heads, int32_t head_dim, int32_t n_tokens, int32_t window,
+                                  int32_t dtype, float* row_stats, void* stream) {
+  if (!q_win || !k || !modality || !row_stats) return MEDA_ERR_INVALID_ARG;
+  if (dtype != MEDA_BF16 && dtype != MEDA_F32) return MEDA_ERR_INVALID_ARG;
+  if (n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads != 0 || n_tokens < 1 || window < 1 ||
+      window > n_tokens || window > kMaxWindow)
+    return MEDA_ERR_SHAPE;
+  if (head_dim != 64 && head_dim != 128 && head_dim != 256) return MEDA_ERR_SHAPE;
+  if ((int64_t)n_q_heads * window > MEDA_STATIC_STATS_MAX_ROWS) return MEDA_ERR_SHAPE;   // beyond the fixed scratch
+  const int smem = attn_generic_smem(window, head_dim, false).total;
+  if (smem > kMaxDynSmem - 4096) return MEDA_ERR_SHAPE;   // leaves room for the kernel's static shared memory
+
+  float* partial = nullptr;
+  meda_status r = static_stats_scratch(&partial);
+  if (r != MEDA_OK) return r;
+
+  cudaStream_t st = as_stream(stream);
+  const int chunks = std::min(kStatsChunks, generic_tiles(n_tokens));
+  const int group = n_q_heads / n_kv_heads;
+  const float scale = 1.0f / sqrtf((float)head_dim);
+  // Every (chunk, head) block writes its whole slice of `partial` before the second kernel reads
+  // it, so what an earlier call left there is never seen.
+  if (dtype == MEDA_F32)
+    stats_partial_kernel<float><<<dim3(chunks, n_q_heads), kAttnThreads, smem, st>>>(
+        static_cast<const float*>(q_win), static_cast<const float*>(k), modality, partial, n_q_heads, group, n_tokens,
+        window, head_dim, scale);
+  else
+    stats_partial_kernel<__nv_bfloat16><<<dim3(chunks, n_q_heads), kAttnThreads, smem, st>>>(
+        static_cast<const __nv_bfloat16*>(q_win), static_cast<const __nv_bfloat16*>(k), modality, partial, n_q_heads,
+        group, n_tokens, window, head_dim, scale);
+  stats_combine_kernel<<<n_q_heads, kMaxWindow, 0, st>>>(partial, row_stats, chunks, n_q_heads, window);
+  return launch_status();
+}
 
 const char* meda_status_string(meda_status status) {
   switch (status) {

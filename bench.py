@@ -31,10 +31,11 @@ UNIT = "token*layers/s"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long_video_128k")
+    ap.add_argument("--layers", type=int, default=0, help="keep only the first N layers (profiling captures); 0 = all")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -106,6 +107,8 @@ def run_reference(args):
         return
     from paper_2502_17599_b200 import workloads as W
     wl = W.WORKLOADS[args.workload]
+    if args.layers > 0:
+        wl = wl.with_(name=f"{wl.name}_first{args.layers}layers", n_layers=min(args.layers, wl.n_layers))
     import numpy  # noqa: F401  (loads BLAS before the thread count is read)
     times = []
     desc = ""
@@ -219,6 +222,8 @@ def run_ours(args):
         dist.barrier()
 
     wl = W.WORKLOADS[args.workload].with_(seed=W.WORKLOADS[args.workload].seed + 1000 * rank)
+    if args.layers > 0:
+        wl = wl.with_(name=f"{wl.name}_first{args.layers}layers", n_layers=min(args.layers, wl.n_layers))
     L = wl.n_layers
     qs, ks, vs = [], [], []
     for l in range(L):
@@ -329,7 +334,7 @@ def run_ours(args):
 
     cpu = None
     if not args.no_cpu_baseline:
-        sec, desc = oracle_sample_seconds(W.WORKLOADS[args.workload])
+        sec, desc = oracle_sample_seconds(wl)
         cpu = {"value": oracle_throughput(wl, sec), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                "sample": desc, "sample_seconds": sec}
 

@@ -43,14 +43,22 @@ sort_hist_kernel(const int32_t* __restrict__ keys, const int32_t* __restrict__ b
   for (int b = lane; b < kSortBins; b += 32) tg[(size_t)b * n_chunks + chunk] = cnt[warp][b];
 }
 
-// In-place exclusive prefix sum of each head's table in (bin, chunk) order.  One block per head.
+// In-place exclusive prefix sum of each head's table in (bin, chunk) order.  One block per head;
+// `len` is a multiple of 4096 (the chunk count is padded to a multiple of 8), so every thread owns
+// a run of len / 1024 entries that is a whole number of 16-byte vectors.
 __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ table, int len) {
   __shared__ int warp_sums[32];
-  int32_t* t = table + (size_t)blockIdx.x * len;
-  const int per = (len + 1023) / 1024;
-  const int begin = min((int)threadIdx.x * per, len), end = min(begin + per, len);
+  int4* t = reinterpret_cast<int4*>(table + (size_t)blockIdx.x * len);
+  const int per = len / 4096;                         // vectors per thread
+  const int begin = (int)threadIdx.x * per;
   int sum = 0;
-  for (int e = begin; e < end; ++e) sum += t[e];
+  for (int e0 = 0; e0 < per; e0 += 8) {
+    int4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = (e0 + u < per) ? t[begin + e0 + u] : make_int4(0, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) sum += x[u].x + x[u].y + x[u].z + x[u].w;
+  }
   const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
   int incl = sum;
 #pragma unroll
@@ -71,10 +79,13 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ t
   }
   __syncthreads();
   int run = warp_sums[warp] + incl - sum;
-  for (int e = begin; e < end; ++e) {
-    int x = t[e];
-    t[e] = run;
-    run += x;
+  for (int e = 0; e < per; ++e) {
+    int4 x = t[begin + e], y;
+    y.x = run; run += x.x;
+    y.y = run; run += x.y;
+    y.z = run; run += x.z;
+    y.w = run; run += x.w;
+    t[begin + e] = y;
   }
 }
 

@@ -565,7 +565,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
                                               (int)StreamShared<SweepPolicy<64>>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
   }
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
-  ctx->sort_chunks = (int)((n + kSortChunk - 1) / kSortChunk);
+  ctx->sort_chunks = (int)((n + kSortChunk - 1) / kSortChunk + 7) / 8 * 8;   // padded: the scan works on whole vectors
   ctx->seg_chunks = (int)((n + kSegChunk - 1) / kSegChunk);
   ctx->sort_passes = n <= kSortBins ? 1 : (n <= (int64_t)kSortBins * kSortBins ? 2 : 3);
   for (int i = 0; i < 2; ++i) {
@@ -603,6 +603,9 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     // that contexts of different shapes can coexist.
     st = c.dtype == MEDA_F32 ? set_generic_attrs<float>() : set_generic_attrs<__nv_bfloat16>();
   }
+  // selection: one cluster per KV head while a head's keys fit the cluster's shared memory
+  ctx->select_cluster = select_cluster_smem(c.n_tokens).total <= kMaxDynSmem;
+  if (st == MEDA_OK && ctx->select_cluster) st = raise_dyn_smem(select_topk_cluster_kernel);
   if (st != MEDA_OK) {
     free_workspace(ws);
     delete ctx;
@@ -726,9 +729,14 @@ meda_status meda_select_topk(meda_ctx* ctx, int32_t layer, const float* scores, 
   if (out_capacity < 1) return MEDA_ERR_WORKSPACE;
   const meda_config& c = ctx->cfg;
   LaunchScope scope(ctx, MEDA_K_SELECT, as_stream(stream));
-  select_topk_kernel<<<c.n_kv_heads, kSelThreads, 0, as_stream(stream)>>>(
-      scores, ctx->ws.modality, budgets + (size_t)layer * 3, idx_conserved, idx_less, c.n_tokens, out_capacity,
-      ctx->ws.status);
+  if (ctx->select_cluster)
+    select_topk_cluster_kernel<<<kSelClusterSize * c.n_kv_heads, kSelThreads, select_cluster_smem(c.n_tokens).total,
+                                 as_stream(stream)>>>(scores, ctx->ws.modality, budgets + (size_t)layer * 3,
+                                                      idx_conserved, idx_less, c.n_tokens, out_capacity, ctx->ws.status);
+  else
+    select_topk_kernel<<<c.n_kv_heads, kSelThreads, 0, as_stream(stream)>>>(
+        scores, ctx->ws.modality, budgets + (size_t)layer * 3, idx_conserved, idx_less, c.n_tokens, out_capacity,
+        ctx->ws.status);
   return launch_status();
 }
 

@@ -4,6 +4,8 @@
 // result does not depend on thread scheduling.  One thread block per KV head.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "meda_common.cuh"
 
 namespace meda {
@@ -110,6 +112,221 @@ select_topk_kernel(const float* __restrict__ scores, const uint8_t* __restrict__
     }
     kept_before += keep_total;
     equal_before += equal_total;
+  }
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// The same selection with one thread-block cluster per KV head, for sequences whose keys fit the
+// cluster's shared memory: the 8 blocks of a cluster each stage one eighth of the head's scores
+// as 32-bit sort keys, so the radix passes read shared memory only; digit histograms are combined
+// across the cluster through distributed shared memory, and the hardware cluster barrier is the
+// only synchronisation between blocks.  Same ranking, same tie-break, same outputs as the
+// single-block kernel above.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSelClusterSize = 8;
+constexpr int kSelBins = 2048;                    // 11-bit digits: 11 + 11 + 10 bits of the score key
+constexpr int kSelPerThread = 4;                  // consecutive tokens per thread in the compaction
+
+struct SelectClusterSmem {
+  int chunk;          // tokens per block
+  int keys_off, hist_off, total_off, misc_off, total;
+};
+__host__ __device__ inline SelectClusterSmem select_cluster_smem(int n) {
+  SelectClusterSmem L;
+  const int step = kSelThreads * kSelPerThread;
+  L.chunk = ((n + kSelClusterSize - 1) / kSelClusterSize + step - 1) / step * step;
+  int off = 0;
+  L.keys_off = off;  off += L.chunk * 4;
+  L.hist_off = off;  off += kSelBins * 4;
+  L.total_off = off; off += kSelBins * 4;
+  L.misc_off = off;  off += 256;
+  L.total = off;
+  return L;
+}
+
+// Exclusive prefix of `v` over the block in thread order, and the block total.  `scratch` holds 33 ints.
+__device__ __forceinline__ int block_exclusive_sum(int v, int* scratch, int& total) {
+  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  __syncthreads();                      // previous users of scratch are done
+  if (lane == 31) scratch[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = scratch[lane], wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += y;
+    }
+    scratch[lane] = wi - w;
+    if (lane == 31) scratch[32] = wi;
+  }
+  __syncthreads();
+  total = scratch[32];
+  return scratch[warp] + incl - v;
+}
+
+__global__ void __cluster_dims__(kSelClusterSize, 1, 1) __launch_bounds__(kSelThreads)
+select_topk_cluster_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ modality,
+                           const int32_t* __restrict__ budget_row, int32_t* __restrict__ idx_conserved,
+                           int32_t* __restrict__ idx_less, int n, int cap, int* status) {
+  namespace cg = cooperative_groups;
+  extern __shared__ __align__(16) unsigned char sel_smem[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const SelectClusterSmem L = select_cluster_smem(n);
+  unsigned int* keys = reinterpret_cast<unsigned int*>(sel_smem + L.keys_off);
+  unsigned int* hist = reinterpret_cast<unsigned int*>(sel_smem + L.hist_off);
+  unsigned int* total = reinterpret_cast<unsigned int*>(sel_smem + L.total_off);
+  int* misc = reinterpret_cast<int*>(sel_smem + L.misc_off);
+  // misc: [0..32] scan scratch, [40] text candidates of this block, [41] kept for sure, [42] equal to the
+  // threshold, [44] digit, [45] remaining
+  const int rank = (int)cluster.block_rank();
+  const int g = blockIdx.x / kSelClusterSize;
+  const int S = budget_row[0], M = budget_row[1], N = budget_row[2];
+  const int n_cand = n - M;
+  if (S < 0 || M < 0 || N < 0 || S != M + N || M > n || N > n_cand || S > cap) {     // uniform over the cluster
+    if (threadIdx.x == 0 && rank == 0) set_status(status, S > cap ? MEDA_ERR_WORKSPACE : MEDA_ERR_BUDGET_INFEASIBLE);
+    return;
+  }
+  const float* sc = scores + (size_t)g * n;
+  int32_t* out_c = idx_conserved + (size_t)g * cap;
+  int32_t* out_l = idx_less + (size_t)g * n;
+  const int lo = rank * L.chunk, hi = min(lo + L.chunk, n);
+
+  // ---- stage the keys; count the text candidates
+  int my_text = 0;
+  for (int j = lo + (int)threadIdx.x; j < hi; j += kSelThreads) {
+    unsigned int b = __float_as_uint(sc[j]);
+    keys[j - lo] = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    my_text += (j < n_cand && modality[j] == MEDA_TEXT) ? 1 : 0;
+  }
+  my_text = __reduce_add_sync(0xffffffffu, my_text);
+  if (threadIdx.x == 0) misc[40] = 0;
+  __syncthreads();
+  if (threadIdx.x % 32 == 0 && my_text) atomicAdd(&misc[40], my_text);
+  cluster.sync();
+  int text_total = 0;
+  for (int r = 0; r < kSelClusterSize; ++r) text_total += cluster.map_shared_rank(misc, r)[40];
+  // Eq. 9 puts every text candidate ahead of every visual one: the N-th ranked candidate is a text
+  // token iff N <= #text candidates; the other class is then wholly kept or wholly dropped.
+  const int cls = (N <= text_total) ? MEDA_TEXT : MEDA_VISUAL;
+  int remaining = (cls == MEDA_TEXT) ? N : N - text_total;
+
+  // ---- the `remaining`-th largest key inside the class, most significant digit first
+  unsigned int prefix = 0u, mask = 0u;
+  if (N > 0) {
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+      const unsigned int bins = pass == 2 ? 1024u : 2048u;
+      for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) hist[b] = 0u;
+      __syncthreads();
+      for (int j = lo + (int)threadIdx.x; j < min(hi, n_cand); j += kSelThreads) {
+        const unsigned int key = keys[j - lo];
+        if (modality[j] == cls && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & (bins - 1u)], 1u);
+      }
+      cluster.sync();                                   // every block's histogram is complete
+      for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) {
+        unsigned int t = 0u;
+#pragma unroll
+        for (int r = 0; r < kSelClusterSize; ++r) t += cluster.map_shared_rank(hist, r)[b];
+        total[b] = t;
+      }
+      cluster.sync();                                   // remote reads are done before the histograms are reused
+      if (threadIdx.x < 32) {
+        // lane l owns bins [64 l, 64 l + 64); walk from the top bin down
+        const int lane = threadIdx.x;
+        int mine = 0;
+        for (int b = 0; b < 64; ++b) mine += (int)total[lane * 64 + b];
+        int above = 0;                                  // keys in bins owned by higher lanes
+        for (int o = 31; o > 0; --o) {
+          int y = __shfl_sync(0xffffffffu, mine, o);
+          if (o > lane) above += y;
+        }
+        if (above < remaining && above + mine >= remaining) {
+          int cum = above;
+          for (int b = 63; b >= 0; --b) {
+            const int c = (int)total[lane * 64 + b];
+            if (cum + c >= remaining) { misc[44] = lane * 64 + b; misc[45] = remaining - cum; break; }
+            cum += c;
+          }
+        }
+      }
+      __syncthreads();
+      prefix |= (unsigned int)misc[44] << shift;
+      mask |= (bins - 1u) << shift;
+      remaining = misc[45];
+      __syncthreads();
+    }
+  }
+  const unsigned int threshold = prefix;
+  const int take_equal = N > 0 ? remaining : 0;
+
+  // ---- classify own tokens: 2 = kept for sure, 1 = equal to the threshold, 0 = dropped
+  auto classify = [&](int j) -> int {
+    if (j >= n) return 0;
+    if (j >= n_cand) return 2;
+    if (N == 0) return 0;
+    const int md = modality[j];
+    if (md != cls) return (cls == MEDA_VISUAL) ? 2 : 0;
+    const unsigned int key = keys[j - lo];
+    return key > threshold ? 2 : (key == threshold ? 1 : 0);
+  };
+  int sure = 0, equal = 0;
+  for (int j = lo + (int)threadIdx.x; j < hi; j += kSelThreads) {
+    const int c = classify(j);
+    sure += c == 2;
+    equal += c == 1;
+  }
+  sure = __reduce_add_sync(0xffffffffu, sure);
+  equal = __reduce_add_sync(0xffffffffu, equal);
+  if (threadIdx.x == 0) { misc[41] = 0; misc[42] = 0; }
+  __syncthreads();
+  if (threadIdx.x % 32 == 0) { atomicAdd(&misc[41], sure); atomicAdd(&misc[42], equal); }
+  cluster.sync();
+  int kept_before = 0, equal_before = 0;
+  for (int r = 0; r < rank; ++r) {
+    const int* m = cluster.map_shared_rank(misc, r);
+    const int e = m[42];
+    kept_before += m[41] + min(max(take_equal - equal_before, 0), e);
+    equal_before += e;
+  }
+  cluster.sync();                                       // nobody reads this block's counters after this point
+
+  // ---- ordered compaction of own tokens, kSelPerThread consecutive tokens per thread
+  for (int base = lo; base < hi; base += kSelThreads * kSelPerThread) {
+    const int j0 = base + (int)threadIdx.x * kSelPerThread;
+    int c[kSelPerThread];
+    int eq = 0;
+#pragma unroll
+    for (int x = 0; x < kSelPerThread; ++x) { c[x] = (j0 + x < hi) ? classify(j0 + x) : 0; eq += c[x] == 1; }
+    int eq_total, keep_total;
+    int eq_rank = equal_before + block_exclusive_sum(eq, misc, eq_total);
+    int keep = 0;
+    bool k[kSelPerThread];
+#pragma unroll
+    for (int x = 0; x < kSelPerThread; ++x) {
+      k[x] = c[x] == 2 || (c[x] == 1 && eq_rank < take_equal);
+      eq_rank += c[x] == 1;
+      keep += k[x];
+    }
+    int pos = kept_before + block_exclusive_sum(keep, misc, keep_total);
+#pragma unroll
+    for (int x = 0; x < kSelPerThread; ++x) {
+      const int j = j0 + x;
+      if (j < hi) {
+        if (k[x]) { out_c[pos] = j; ++pos; }
+        else out_l[j - pos] = j;
+      }
+    }
+    kept_before += keep_total;
+    equal_before += eq_total;
   }
 }
 

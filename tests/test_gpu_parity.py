@@ -288,3 +288,27 @@ def test_contexts_of_different_shapes_coexist():
     P.assert_scores_close(P.np64(buf.scores), O.window_scores(qh, kh))
     ctx_small.close()
     ctx_big.close()
+
+
+def test_select_beyond_cluster_capacity_uses_the_single_block_kernel():
+    """A head whose keys do not fit one cluster's shared memory (n > 393,216) is selected by the
+    single-block kernel; same ranking and tie-break."""
+    n = 400_003
+    wl = W.small_variant("select_400k", dtype="f32", n_layers=1, n_q_heads=1, n_kv_heads=1, head_dim=64, window=8,
+                         spans=((0, 1000, 0), (1000, n - 500, 1), (n - 500, n, 0)), rho=0.1, frame_tokens=0)
+    ctx = make_ctx(wl)
+    rng = np.random.default_rng(5)
+    a_s = rng.random(n).astype(np.float32)
+    a_s[1234:1300] = a_s[1234]                      # a run of exact ties
+    mod = wl.modality().numpy()
+    scores = torch.from_numpy(a_s[None]).cuda()
+    idx_c = torch.full((1, n), -1, dtype=torch.int32, device="cuda")
+    idx_l = torch.full((1, n), -1, dtype=torch.int32, device="cuda")
+    for M, N in ((3000, 1040), (10, 2000)):
+        budgets = torch.tensor([[M + N, M, N]], dtype=torch.int32, device="cuda")
+        ctx.select_topk(0, scores, budgets, idx_c, idx_l, n)
+        ctx.check()
+        assert P.compare_selection(idx_c[0, : M + N].cpu().numpy(), a_s.astype(np.float64), mod, M, N) == 0
+        less = idx_l[0, : n - M - N].cpu().numpy()
+        assert (np.diff(less) > 0).all() and less.size + M + N == n
+    ctx.close()

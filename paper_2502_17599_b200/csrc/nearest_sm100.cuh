@@ -68,8 +68,14 @@ struct NearestPolicy {
     const int S = slots(p);
     return S > 0 && S < p.n;                       // otherwise there is nothing to merge
   }
+  // Token rows [n - M, n) are the recent window: always conserved, never merged, so the 256-row
+  // blocks that lie wholly inside it are not swept.
+  __device__ static int rows_swept(const Params& p) {
+    const int m = min(max(p.budget_row[1], 0), p.n);
+    return p.n - m;
+  }
   __device__ static bool get_item(const Params& p, int it, StreamItem& o) {
-    const int m_blocks = (p.n + 255) / 256;
+    const int m_blocks = (rows_swept(p) + 255) / 256;
     const int idx = blockIdx.x + it * gridDim.x;
     if (idx >= m_blocks * p.n_heads) return false;
     const int S = slots(p);
@@ -98,6 +104,39 @@ struct NearestPolicy {
       best = -INFINITY;
       best_slot = 0;
     }
+    // One chunk = this thread's row against 32 consecutive slots: scale by the slots' inverse norms
+    // (two products per instruction), reduce with three-input maxima, and only when the chunk
+    // beats the running best look for the first slot that attains it.
+    __device__ __forceinline__ void chunk(const uint32_t (&r)[32], int chunk_idx, int c0, int S, bool ragged) {
+      const ulonglong2* inv2 = reinterpret_cast<const ulonglong2*>(inv_t + chunk_idx * 32);
+      float v[32];
+#pragma unroll
+      for (int x = 0; x < 8; ++x) {
+        const ulonglong2 w = inv2[x];
+        sm100::mul_f32x2(sm100::pack_f32x2(r[4 * x + 0], r[4 * x + 1]), w.x, v[4 * x + 0], v[4 * x + 1]);
+        sm100::mul_f32x2(sm100::pack_f32x2(r[4 * x + 2], r[4 * x + 3]), w.y, v[4 * x + 2], v[4 * x + 3]);
+      }
+      const int s0 = c0 + chunk_idx * 32;
+      if (ragged) {
+#pragma unroll
+        for (int x = 0; x < 32; ++x) if (s0 + x >= S) v[x] = -INFINITY;
+      }
+      float t[12];
+#pragma unroll
+      for (int x = 0; x < 10; ++x) t[x] = sm100::fmax3(v[3 * x], v[3 * x + 1], v[3 * x + 2]);
+      t[10] = v[30];
+      t[11] = v[31];
+      const float u0 = sm100::fmax3(t[0], t[1], t[2]), u1 = sm100::fmax3(t[3], t[4], t[5]);
+      const float u2 = sm100::fmax3(t[6], t[7], t[8]), u3 = sm100::fmax3(t[9], t[10], t[11]);
+      const float cmax = fmaxf(sm100::fmax3(u0, u1, u2), u3);
+      if (cmax > best) {
+        int first = 31;
+#pragma unroll
+        for (int x = 30; x >= 0; --x) if (v[x] == cmax) first = x;
+        best = cmax;
+        best_slot = s0 + first;
+      }
+    }
     __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
       const int S = it.u0;
       const int c0 = tile * 128;
@@ -108,31 +147,24 @@ struct NearestPolicy {
       reinterpret_cast<float4*>(inv_t)[lane] = __ldg(reinterpret_cast<const float4*>(inv_g + c0) + lane);
       __syncwarp();
       const bool ragged = c0 + 128 > S;
-#pragma unroll 1
-      for (int chunk = 0; chunk < 4; ++chunk) {
-        float v[32];
-        sm100::tmem_ld_32x32(taddr + chunk * 32u, v);
-        const float4* inv4 = reinterpret_cast<const float4*>(inv_t + chunk * 32);
-#pragma unroll
-        for (int x = 0; x < 8; ++x) {
-          const float4 w = inv4[x];
-          v[4 * x + 0] *= w.x; v[4 * x + 1] *= w.y; v[4 * x + 2] *= w.z; v[4 * x + 3] *= w.w;
-        }
-        if (ragged) {
-#pragma unroll
-          for (int x = 0; x < 32; ++x) if (c0 + chunk * 32 + x >= S) v[x] = -INFINITY;
-        }
-        float cmax = -INFINITY;
-#pragma unroll
-        for (int x = 0; x < 32; ++x) cmax = fmaxf(cmax, v[x]);
-        if (cmax > best) {
-          int first = 31;
-#pragma unroll
-          for (int x = 31; x >= 0; --x) if (v[x] == cmax) first = x;
-          best = cmax;
-          best_slot = c0 + chunk * 32 + first;
-        }
-      }
+      // two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced
+      uint32_t ra[32], rb[32];
+      sm100::tmem_ld_32x32_issue(taddr, ra);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(ra);
+      sm100::tmem_ld_32x32_issue(taddr + 32u, rb);
+      chunk(ra, 0, c0, S, ragged);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(rb);
+      sm100::tmem_ld_32x32_issue(taddr + 64u, ra);
+      chunk(rb, 1, c0, S, ragged);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(ra);
+      sm100::tmem_ld_32x32_issue(taddr + 96u, rb);
+      chunk(ra, 2, c0, S, ragged);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(rb);
+      chunk(rb, 3, c0, S, ragged);
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {
       const int token = it.a_row + row_in_block;

@@ -118,19 +118,33 @@ stats_partial_kernel(const T* __restrict__ q_win, const T* __restrict__ k, const
   for (int e = threadIdx.x; e < w * 4; e += blockDim.x) out[e] = rs[e / 4][e % 4];
 }
 
-// row_stats[h][i] = merge over chunks, in chunk order.  grid = Hq, block = kMaxWindow.
-__global__ void stats_combine_kernel(const float* __restrict__ partial, float* __restrict__ row_stats,
-                                     int chunks, int hq, int w) {
-  const int h = blockIdx.x, i = threadIdx.x;
-  if (i >= w) return;
+// row_stats[row] = merge over the key chunks' partial normalisers, row = h * w + i.  One warp per row:
+// lane l merges chunks l, l + 32, ... in order, then the lanes are merged pairwise in a fixed
+// butterfly, so the result does not depend on scheduling.  grid = ceil(rows / 8), block = 256.
+__global__ void __launch_bounds__(256)
+stats_combine_kernel(const float* __restrict__ partial, float* __restrict__ row_stats, int chunks, int rows) {
+  const int row = blockIdx.x * 8 + threadIdx.x / 32, lane = threadIdx.x % 32;
+  if (row >= rows) return;
   float m = -INFINITY, z = 0.f, mv = -INFINITY, zv = 0.f;
-  for (int c = 0; c < chunks; ++c) {
-    const float* p = partial + (((size_t)c * hq + h) * w + i) * 4;
-    merge_mz(m, z, p[0], p[1]);
-    merge_mz(mv, zv, p[2], p[3]);
+  for (int c = lane; c < chunks; c += 32) {
+    const float4 p = reinterpret_cast<const float4*>(partial)[(size_t)c * rows + row];
+    merge_mz(m, z, p.x, p.y);
+    merge_mz(mv, zv, p.z, p.w);
   }
-  float* o = row_stats + ((size_t)h * w + i) * 4;
-  o[0] = m; o[1] = z; o[2] = mv; o[3] = zv;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), z2 = __shfl_xor_sync(0xffffffffu, z, o);
+    const float mv2 = __shfl_xor_sync(0xffffffffu, mv, o), zv2 = __shfl_xor_sync(0xffffffffu, zv, o);
+    // both partners must compute the same bits: merge in (lower lane, higher lane) order
+    const bool low = (lane & o) == 0;
+    float ma = low ? m : m2, za = low ? z : z2, mb = low ? m2 : m, zb = low ? z2 : z;
+    merge_mz(ma, za, mb, zb);
+    m = ma; z = za;
+    float mva = low ? mv : mv2, zva = low ? zv : zv2, mvb = low ? mv2 : mv, zvb = low ? zv2 : zv;
+    merge_mz(mva, zva, mvb, zvb);
+    mv = mva; zv = zva;
+  }
+  if (lane == 0) reinterpret_cast<float4*>(row_stats)[row] = make_float4(m, z, mv, zv);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -16,31 +16,31 @@ namespace meda {
 
 constexpr int kSortBits = 9;
 constexpr int kSortBins = 1 << kSortBits;
-constexpr int kSortChunk = 1024;      // elements ranked by one warp
 constexpr int kSortWarps = 8;
+constexpr int kSortWarpItems = 256;                          // elements ranked by one warp
+constexpr int kSortBlockItems = kSortWarps * kSortWarpItems; // elements of one block = one column of the digit table
 constexpr int kSegChunk = 128;        // sorted rows walked by one warp
 constexpr int kSegWarps = 8;
 
 // ---- stable radix pass: histogram, scan, scatter ----------------------------------------------
-// table[g][bin][chunk] <- number of keys of warp-chunk `chunk` whose digit is `bin`.
+// table[g][bin][block] <- number of keys of block `block` whose digit is `bin`.
 __global__ void __launch_bounds__(kSortWarps * 32)
 sort_hist_kernel(const int32_t* __restrict__ keys, const int32_t* __restrict__ budget_row, int32_t* __restrict__ table,
-                 int n, int cap, int shift, int n_chunks) {
-  __shared__ int cnt[kSortWarps][kSortBins];
-  const int g = blockIdx.y, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int chunk = blockIdx.x * kSortWarps + warp;
-  if (chunk >= n_chunks) return;
+                 int n, int cap, int shift, int n_blocks) {
+  __shared__ int cnt[kSortBins];
+  const int g = blockIdx.y, blk = blockIdx.x;
   const int n_less = n - min(budget_row[0], cap);
-  for (int b = lane; b < kSortBins; b += 32) cnt[warp][b] = 0;
-  __syncwarp();
+  for (int b = threadIdx.x; b < kSortBins; b += blockDim.x) cnt[b] = 0;
+  __syncthreads();
   const int32_t* kg = keys + (size_t)g * n;
-  for (int r = 0; r < kSortChunk / 32; ++r) {
-    int q = chunk * kSortChunk + r * 32 + lane;
-    if (q < n_less) atomicAdd(&cnt[warp][(kg[q] >> shift) & (kSortBins - 1)], 1);
+#pragma unroll
+  for (int r = 0; r < kSortBlockItems / (kSortWarps * 32); ++r) {
+    const int q = blk * kSortBlockItems + r * (kSortWarps * 32) + (int)threadIdx.x;
+    if (q < n_less) atomicAdd(&cnt[(kg[q] >> shift) & (kSortBins - 1)], 1);
   }
-  __syncwarp();
-  int32_t* tg = table + (size_t)g * kSortBins * n_chunks;
-  for (int b = lane; b < kSortBins; b += 32) tg[(size_t)b * n_chunks + chunk] = cnt[warp][b];
+  __syncthreads();
+  int32_t* tg = table + (size_t)g * kSortBins * n_blocks;
+  for (int b = threadIdx.x; b < kSortBins; b += blockDim.x) tg[(size_t)b * n_blocks + blk] = cnt[b];
 }
 
 // In-place exclusive prefix sum of each head's table in (bin, chunk) order.  One block per head;
@@ -89,32 +89,53 @@ __global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ t
   }
 }
 
-// Stable scatter of (key, row) pairs by the digit at `shift`, using the scanned table.
+// Stable scatter of (key, row) pairs by the digit at `shift`, using the scanned table.  Inside a block
+// the eight warps own consecutive runs of 256 elements: each first counts its digits, the counts are
+// turned into per-warp start offsets (block base from the table + the earlier warps' counts), then every
+// warp ranks its elements in index order.
 __global__ void __launch_bounds__(kSortWarps * 32)
 sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restrict__ rows_in,
                     const int32_t* __restrict__ budget_row, const int32_t* __restrict__ table,
                     int32_t* __restrict__ keys_out, int32_t* __restrict__ rows_out, int n, int cap, int shift,
-                    int n_chunks) {
+                    int n_blocks) {
   __shared__ int cnt[kSortWarps][kSortBins];
-  const int g = blockIdx.y, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int chunk = blockIdx.x * kSortWarps + warp;
-  if (chunk >= n_chunks) return;
+  const int g = blockIdx.y, blk = blockIdx.x, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int n_less = n - min(budget_row[0], cap);
-  if (chunk * kSortChunk >= n_less) return;
-  const int32_t* tg = table + (size_t)g * kSortBins * n_chunks;
-  for (int b = lane; b < kSortBins; b += 32) cnt[warp][b] = tg[(size_t)b * n_chunks + chunk];
-  __syncwarp();
+  if (blk * kSortBlockItems >= n_less) return;            // uniform over the block
   const int32_t* kg = keys_in + (size_t)g * n;
   const int32_t* rg = rows_in + (size_t)g * n;
   int32_t* ko = keys_out + (size_t)g * n;
   int32_t* ro = rows_out + (size_t)g * n;
+  const int q0 = blk * kSortBlockItems + warp * kSortWarpItems;
+  constexpr int kRounds = kSortWarpItems / 32;
+  int key[kRounds];
+  for (int b = lane; b < kSortBins; b += 32) cnt[warp][b] = 0;
+  __syncwarp();
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int q = q0 + r * 32 + lane;
+    key[r] = q < n_less ? kg[q] : -1;
+    if (key[r] >= 0) atomicAdd(&cnt[warp][(key[r] >> shift) & (kSortBins - 1)], 1);
+  }
+  __syncthreads();
+  const int32_t* tg = table + (size_t)g * kSortBins * n_blocks;
+  for (int b = threadIdx.x; b < kSortBins; b += blockDim.x) {
+    int run = tg[(size_t)b * n_blocks + blk];
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) {
+      const int c = cnt[w][b];
+      cnt[w][b] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
   const unsigned int lt = (1u << lane) - 1u;
-  for (int r = 0; r < kSortChunk / 32; ++r) {
-    const int q = chunk * kSortChunk + r * 32 + lane;
-    const bool valid = q < n_less;
-    const int key = valid ? kg[q] : 0;
+#pragma unroll
+  for (int r = 0; r < kRounds; ++r) {
+    const int q = q0 + r * 32 + lane;
+    const bool valid = key[r] >= 0;
+    const int digit = (key[r] >> shift) & (kSortBins - 1);
     const int row = valid ? rg[q] : 0;
-    const int digit = (key >> shift) & (kSortBins - 1);
     const unsigned int peers = __match_any_sync(0xffffffffu, valid ? digit : kSortBins + lane);
     const int leader = __ffs(peers) - 1;
     int base = 0;
@@ -125,7 +146,7 @@ sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restri
     base = __shfl_sync(0xffffffffu, base, leader);
     if (valid) {
       const int pos = min(base + __popc(peers & lt), n - 1);
-      ko[pos] = key;
+      ko[pos] = key[r];
       ro[pos] = row;
     }
     __syncwarp();
@@ -287,8 +308,8 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
   constexpr int E = D / 32;
   const int g = blockIdx.y, lane = threadIdx.x % 32;
   const int S = min(budget_row[0], cap);
-  const int slot = blockIdx.x * 8 + threadIdx.x / 32;
-  if (slot >= S) return;
+  // the grid is sized on the host for the largest possible S: walk the slots with a stride
+  for (int slot = blockIdx.x * 8 + threadIdx.x / 32; slot < S; slot += gridDim.x * 8) {
   const int start = evict ? 0 : seg_start[(size_t)g * n + slot];
   const int end = evict ? 0 : seg_end[(size_t)g * n + slot];
   float ak[E], av[E];
@@ -299,7 +320,7 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
     load_row<T, E>(v + ((size_t)g * n + own) * D, lane, av);
   } else {
     const int c0 = start / kSegChunk, c1 = (end - 1) / kSegChunk;
-    if (c0 == c1) return;
+    if (c0 == c1) continue;
     float* base = const_cast<float*>(carry);
     const float* p = carry_ptr<D>(base, g, c0, 1, n_chunks);
 #pragma unroll
@@ -316,6 +337,7 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
   store_row<T, E>(k_out + ((size_t)g * cap + slot) * D, lane, ak, c);
   store_row<T, E>(v_out + ((size_t)g * cap + slot) * D, lane, av, c);
   if (lane == 0) counts[(size_t)g * cap + slot] = members + 1;
+  }
 }
 
 // Clears the per-slot segment bounds of one layer (slots without members must read as empty).
@@ -323,8 +345,10 @@ __global__ void clear_segments_kernel(int32_t* __restrict__ seg_start, int32_t* 
                                       const int32_t* __restrict__ budget_row, int n, int cap) {
   const int g = blockIdx.y;
   const int S = min(budget_row[0], cap);
-  const int s = blockIdx.x * blockDim.x + threadIdx.x;
-  if (s < S) { seg_start[(size_t)g * n + s] = 0; seg_end[(size_t)g * n + s] = 0; }
+  for (int s = blockIdx.x * blockDim.x + threadIdx.x; s < S; s += gridDim.x * blockDim.x) {
+    seg_start[(size_t)g * n + s] = 0;
+    seg_end[(size_t)g * n + s] = 0;
+  }
 }
 
 }  // namespace meda

@@ -164,7 +164,8 @@ meda_status launch_stats(meda_ctx* ctx, const void* q_win, const void* k, float*
   }
   {
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
-    stats_combine_kernel<<<c.n_q_heads, kMaxWindow, 0, st>>>(ctx->ws.stats_partial, row_stats, chunks, c.n_q_heads, c.window);
+    stats_combine_kernel<<<(c.n_q_heads * c.window + 7) / 8, 256, 0, st>>>(ctx->ws.stats_partial, row_stats, chunks,
+                                                                               c.n_q_heads * c.window);
   }
   return launch_status();
 }
@@ -216,7 +217,8 @@ meda_status launch_stats_fast(meda_ctx* ctx, const void* q_win, const void* k, f
   }
   {
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
-    stats_combine_kernel<<<c.n_q_heads, kMaxWindow, 0, st>>>(ctx->ws.stats_partial, row_stats, prm.chunks, c.n_q_heads, c.window);
+    stats_combine_kernel<<<(c.n_q_heads * c.window + 7) / 8, 256, 0, st>>>(ctx->ws.stats_partial, row_stats, prm.chunks,
+                                                                               c.n_q_heads * c.window);
   }
   return launch_status();
 }
@@ -280,7 +282,7 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
   const int max_slots = std::min(cap, n);
   {
     LaunchScope scope(ctx, MEDA_K_PREP, st);
-    gather_conserved_bf16_kernel<<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
+    gather_conserved_bf16_kernel<<<dim3(std::min((max_slots + 7) / 8, ctx->sm_count * 8), c.n_kv_heads), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(k), idx_conserved, budget_row, ctx->ws.kc, ctx->ws.inv_norm, n, cap,
         ctx->kc_rows, ctx->inv_stride);
   }
@@ -315,7 +317,7 @@ void launch_seg_kernels(meda_ctx* ctx, const void* k, const void* v, const int32
         ctx->ws.carry_cnt, n, cap, ctx->seg_chunks);
   }
   LaunchScope scope(ctx, MEDA_K_REDUCE, st);
-  seg_finalize_kernel<T, D><<<dim3((max_slots + 7) / 8, c.n_kv_heads), 256, 0, st>>>(
+  seg_finalize_kernel<T, D><<<dim3(std::min((max_slots + 7) / 8, ctx->sm_count * 8), c.n_kv_heads), 256, 0, st>>>(
       static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, budget_row, ctx->ws.seg_start,
       ctx->ws.seg_end, ctx->ws.carry, ctx->ws.carry_cnt, static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n,
       cap, ctx->seg_chunks, evict);
@@ -334,10 +336,10 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
   if (!evict) {
     {
       LaunchScope scope(ctx, MEDA_K_GROUP, st);
-      clear_segments_kernel<<<dim3((max_slots + 255) / 256, c.n_kv_heads), 256, 0, st>>>(ctx->ws.seg_start,
+      clear_segments_kernel<<<dim3(std::min((max_slots + 255) / 256, ctx->sm_count), c.n_kv_heads), 256, 0, st>>>(ctx->ws.seg_start,
                                                                                        ctx->ws.seg_end, budget_row, n, cap);
     }
-    const dim3 grid((ctx->sort_chunks + kSortWarps - 1) / kSortWarps, c.n_kv_heads);
+    const dim3 grid(ctx->sort_chunks, c.n_kv_heads);
     for (int pass = 0; pass < ctx->sort_passes; ++pass) {
       int32_t* ko = ctx->ws.sort_keys[pass & 1];
       int32_t* ro = ctx->ws.sort_rows[pass & 1];
@@ -472,7 +474,7 @@ meda_status meda_row_stats_static(const void* q_win, const void* k, const uint8_
     stats_partial_kernel<__nv_bfloat16><<<dim3(chunks, n_q_heads), kAttnThreads, smem, st>>>(
         static_cast<const __nv_bfloat16*>(q_win), static_cast<const __nv_bfloat16*>(k), modality, partial, n_q_heads,
         group, n_tokens, window, head_dim, scale);
-  stats_combine_kernel<<<n_q_heads, kMaxWindow, 0, st>>>(partial, row_stats, chunks, n_q_heads, window);
+  stats_combine_kernel<<<(n_q_heads * window + 7) / 8, 256, 0, st>>>(partial, row_stats, chunks, n_q_heads * window);
   return launch_status();
 }
 
@@ -565,7 +567,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
                                               (int)StreamShared<SweepPolicy<64>>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
   }
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
-  ctx->sort_chunks = (int)((n + kSortChunk - 1) / kSortChunk + 7) / 8 * 8;   // padded: the scan works on whole vectors
+  ctx->sort_chunks = (int)((n + kSortBlockItems - 1) / kSortBlockItems + 7) / 8 * 8;   // padded: the scan works on whole vectors
   ctx->seg_chunks = (int)((n + kSegChunk - 1) / kSegChunk);
   ctx->sort_passes = n <= kSortBins ? 1 : (n <= (int64_t)kSortBins * kSortBins ? 2 : 3);
   for (int i = 0; i < 2; ++i) {

@@ -28,7 +28,7 @@ struct Workspace {
   int32_t* token_target = nullptr;    // [Hkv][n] nearest slot of every token row (tensor-core path)
   int32_t* sort_keys[2] = {nullptr, nullptr};   // [Hkv][n] ping-pong: target slot of each sorted entry
   int32_t* sort_rows[2] = {nullptr, nullptr};   // [Hkv][n] ping-pong: token row of each sorted entry
-  int32_t* sort_table = nullptr;      // [Hkv][bins][sort_chunks] digit counts, then offsets
+  int32_t* sort_table = nullptr;      // [Hkv][bins][sort blocks] digit counts, then offsets
   int32_t* seg_start = nullptr;       // [Hkv][n] first sorted position of each slot's members
   int32_t* seg_end = nullptr;         // [Hkv][n] one past the last
   float* carry = nullptr;             // [Hkv][seg_chunks][2][2 * d] partial sums of slots that cross chunk borders
@@ -63,7 +63,7 @@ struct meda_ctx {
   int ent_slots = 0;      // entries of ent_partial written by one entropy sweep
   int inv_stride = 0;     // floats per head in ws.inv_norm (padded so 128-wide slices can be read whole)
   int kc_rows = 0;        // rows per head in ws.kc
-  int sort_chunks = 0;    // warp-chunks per head in the grouping sort
+  int sort_chunks = 0;    // blocks per head in the grouping sort (columns of its digit table)
   int seg_chunks = 0;     // warp-chunks per head in the segmented average
   int sort_passes = 1;    // 9-bit digit passes needed to order slots < n_tokens
   bool fast = false;      // bf16 with head_dim 128: tensor-core kernels are used

@@ -23,19 +23,20 @@ gather_conserved_bf16_kernel(const __nv_bfloat16* __restrict__ k, const int32_t*
                              float* __restrict__ inv_norm, int n, int cap, int kc_rows, int inv_stride) {
   const int g = blockIdx.y;
   const int S = min(budget_row[0], cap);
-  const int slot = blockIdx.x * 8 + threadIdx.x / 32;
-  if (slot >= S) return;
   const int lane = threadIdx.x % 32;
-  int row = idx_conserved[(size_t)g * cap + slot];
-  row = min(max(row, 0), n - 1);
-  const uint2* src = reinterpret_cast<const uint2*>(k + ((size_t)g * n + row) * kFastDim);
-  uint2 x = src[lane];
-  reinterpret_cast<uint2*>(kc + ((size_t)g * kc_rows + slot) * kFastDim)[lane] = x;
-  float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&x.x));
-  float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&x.y));
-  float ss = a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y;
-  ss = warp_sum(ss);
-  if (lane == 0) inv_norm[(size_t)g * inv_stride + slot] = 1.f / fmaxf(sqrtf(ss), kCosEps);
+  // the grid is sized on the host for the largest possible S: walk the slots with a stride
+  for (int slot = blockIdx.x * 8 + threadIdx.x / 32; slot < S; slot += gridDim.x * 8) {
+    int row = idx_conserved[(size_t)g * cap + slot];
+    row = min(max(row, 0), n - 1);
+    const uint2* src = reinterpret_cast<const uint2*>(k + ((size_t)g * n + row) * kFastDim);
+    uint2 x = src[lane];
+    reinterpret_cast<uint2*>(kc + ((size_t)g * kc_rows + slot) * kFastDim)[lane] = x;
+    float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&x.x));
+    float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&x.y));
+    float ss = a.x * a.x + a.y * a.y + b.x * b.x + b.y * b.y;
+    ss = warp_sum(ss);
+    if (lane == 0) inv_norm[(size_t)g * inv_stride + slot] = 1.f / fmaxf(sqrtf(ss), kCosEps);
+  }
 }
 
 // target[g][p] = token_target[g][less[p]]: from per-token results to the less-important list order.

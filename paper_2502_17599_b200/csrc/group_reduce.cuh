@@ -208,8 +208,10 @@ __device__ __forceinline__ void store_row(T* p, int lane, const float (&x)[E], f
   for (int e = 0; e < E; ++e) p[lane * E + e] = from_f32<T>(x[e] / count);
 }
 
+// grid = (chunks / kSegWarps, heads, 2): blockIdx.z picks the tensor (0 keys, 1 values), so that twice
+// as many warps keep rows in flight; the z = 0 warps also record segment bounds and counts.
 template <typename T, int D>
-__global__ void __launch_bounds__(kSegWarps * 32)
+__global__ void __launch_bounds__(kSegWarps * 32, 3)
 seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ keys,
                   const int32_t* __restrict__ rows, const int32_t* __restrict__ idx_conserved,
                   const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,
@@ -217,6 +219,8 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
                   float* __restrict__ carry, int32_t* __restrict__ carry_cnt, int n, int cap, int n_chunks) {
   constexpr int E = D / 32;
   const int g = blockIdx.y, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int tensor = blockIdx.z;
+  const bool book = tensor == 0 && lane == 0;            // the one lane that writes bounds and counts
   const int chunk = blockIdx.x * kSegWarps + warp;
   const int S = min(budget_row[0], cap);
   const int n_less = n - S;
@@ -225,13 +229,13 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
   const int q1 = min(q0 + kSegChunk, n_less);
   const int32_t* kg = keys + (size_t)g * n;
   const int32_t* rg = rows + (size_t)g * n;
-  const T* k_g = k + (size_t)g * n * D;
-  const T* v_g = v + (size_t)g * n * D;
+  const T* x_g = (tensor == 0 ? k : v) + (size_t)g * n * D;
+  T* out_g = (tensor == 0 ? k_out : v_out) + (size_t)g * cap * D;
   const int32_t* cons = idx_conserved + (size_t)g * cap;
   int32_t* st = seg_start + (size_t)g * n;
   int32_t* en = seg_end + (size_t)g * n;
 
-  float ak[E], av[E];
+  float acc[E];
   int members = 0;
   int cur = min(max(kg[q0], 0), S - 1);
   bool started_here = (q0 == 0) || (kg[q0 - 1] != kg[q0]);
@@ -240,54 +244,64 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
     members = 0;
     if (fresh) {
       const int own = min(max(cons[slot], 0), n - 1);
-      load_row<T, E>(k_g + (size_t)own * D, lane, ak);
-      load_row<T, E>(v_g + (size_t)own * D, lane, av);
-      if (lane == 0) st[slot] = q;
+      load_row<T, E>(x_g + (size_t)own * D, lane, acc);
+      if (book) st[slot] = q;
     } else {
 #pragma unroll
-      for (int e = 0; e < E; ++e) { ak[e] = 0.f; av[e] = 0.f; }
+      for (int e = 0; e < E; ++e) acc[e] = 0.f;
     }
   };
   auto end_piece = [&](int slot, bool fresh, bool ended, int q_end) {
-    if (ended && lane == 0) en[slot] = q_end;
+    if (ended && book) en[slot] = q_end;
     if (fresh && ended) {
-      const float c = (float)(members + 1);
-      store_row<T, E>(k_out + ((size_t)g * cap + slot) * D, lane, ak, c);
-      store_row<T, E>(v_out + ((size_t)g * cap + slot) * D, lane, av, c);
-      if (lane == 0) counts[(size_t)g * cap + slot] = members + 1;
+      store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)(members + 1));
+      if (book) counts[(size_t)g * cap + slot] = members + 1;
     } else {
       const int which = fresh ? 1 : 0;
-      float* cp = carry_ptr<D>(carry, g, chunk, which, n_chunks);
+      float* cp = carry_ptr<D>(carry, g, chunk, which, n_chunks) + tensor * D;
 #pragma unroll
-      for (int e = 0; e < E; ++e) { cp[lane * E + e] = ak[e]; cp[D + lane * E + e] = av[e]; }
-      if (lane == 0) carry_cnt[((size_t)g * n_chunks + chunk) * 2 + which] = members;
+      for (int e = 0; e < E; ++e) cp[lane * E + e] = acc[e];
+      if (book) carry_cnt[((size_t)g * n_chunks + chunk) * 2 + which] = members;
     }
   };
 
   begin_segment(cur, started_here, q0);
-  constexpr int kBatch = 8;
+  constexpr int kBatch = 32 / E;                    // 32 row elements per lane in flight
+  // the (slot, row) pairs of the next batch are fetched while the rows of this one are in flight
+  int key[kBatch], row[kBatch];
+#pragma unroll
+  for (int b = 0; b < kBatch; ++b) {
+    const int q = min(q0 + b, q1 - 1);
+    key[b] = kg[q];
+    row[b] = rg[q];
+  }
   for (int qb = q0; qb < q1; qb += kBatch) {
-    float xk[kBatch][E], xv[kBatch][E];
-    int key[kBatch];
+    float x[kBatch][E];
+    int key_now[kBatch];
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
-      const int q = min(qb + b, q1 - 1);
-      key[b] = min(max(kg[q], 0), S - 1);
-      const int row = min(max(rg[q], 0), n - 1);
-      load_row<T, E>(k_g + (size_t)row * D, lane, xk[b]);
-      load_row<T, E>(v_g + (size_t)row * D, lane, xv[b]);
+      key_now[b] = min(max(key[b], 0), S - 1);
+      load_row<T, E>(x_g + (size_t)min(max(row[b], 0), n - 1) * D, lane, x[b]);
+    }
+    if (qb + kBatch < q1) {
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) {
+        const int q = min(qb + kBatch + b, q1 - 1);
+        key[b] = kg[q];
+        row[b] = rg[q];
+      }
     }
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
       if (qb + b < q1) {
-        if (key[b] != cur) {
+        if (key_now[b] != cur) {
           end_piece(cur, started_here, true, qb + b);
-          cur = key[b];
+          cur = key_now[b];
           started_here = true;
           begin_segment(cur, true, qb + b);
         }
 #pragma unroll
-        for (int e = 0; e < E; ++e) { ak[e] += xk[b][e]; av[e] += xv[b][e]; }
+        for (int e = 0; e < E; ++e) acc[e] += x[b][e];
         ++members;
       }
     }
@@ -296,8 +310,9 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
   end_piece(cur, started_here, ended, q1);
 }
 
-// One warp per conserved slot: slots without members are copied, slots whose members span several
-// chunks get their parked pieces added in chunk order; everything else was finished by the walker.
+// One warp per (conserved slot, tensor): slots without members are copied, slots whose members span
+// several chunks get their parked pieces added in chunk order (loaded eight at a time, added one by
+// one); everything else was finished by the walker.  grid = (blocks, heads, 2).
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ idx_conserved,
@@ -307,36 +322,50 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
                     int32_t* __restrict__ counts, int n, int cap, int n_chunks, int evict) {
   constexpr int E = D / 32;
   const int g = blockIdx.y, lane = threadIdx.x % 32;
+  const int tensor = blockIdx.z;
+  const T* x_g = (tensor == 0 ? k : v) + (size_t)g * n * D;
+  T* out_g = (tensor == 0 ? k_out : v_out) + (size_t)g * cap * D;
   const int S = min(budget_row[0], cap);
   // the grid is sized on the host for the largest possible S: walk the slots with a stride
   for (int slot = blockIdx.x * 8 + threadIdx.x / 32; slot < S; slot += gridDim.x * 8) {
-  const int start = evict ? 0 : seg_start[(size_t)g * n + slot];
-  const int end = evict ? 0 : seg_end[(size_t)g * n + slot];
-  float ak[E], av[E];
-  int members = 0;
-  if (end <= start) {
-    const int own = min(max(idx_conserved[(size_t)g * cap + slot], 0), n - 1);
-    load_row<T, E>(k + ((size_t)g * n + own) * D, lane, ak);
-    load_row<T, E>(v + ((size_t)g * n + own) * D, lane, av);
-  } else {
-    const int c0 = start / kSegChunk, c1 = (end - 1) / kSegChunk;
-    if (c0 == c1) continue;
-    float* base = const_cast<float*>(carry);
-    const float* p = carry_ptr<D>(base, g, c0, 1, n_chunks);
+    const int start = evict ? 0 : seg_start[(size_t)g * n + slot];
+    const int end = evict ? 0 : seg_end[(size_t)g * n + slot];
+    float acc[E];
+    int members = 0;
+    if (end <= start) {
+      const int own = min(max(idx_conserved[(size_t)g * cap + slot], 0), n - 1);
+      load_row<T, E>(x_g + (size_t)own * D, lane, acc);
+    } else {
+      const int c0 = start / kSegChunk, c1 = (end - 1) / kSegChunk;
+      if (c0 == c1) continue;
+      float* base = const_cast<float*>(carry);
+      const float* p = carry_ptr<D>(base, g, c0, 1, n_chunks) + tensor * D;
 #pragma unroll
-    for (int e = 0; e < E; ++e) { ak[e] = p[lane * E + e]; av[e] = p[D + lane * E + e]; }
-    members = carry_cnt[((size_t)g * n_chunks + c0) * 2 + 1];
-    for (int c = c0 + 1; c <= c1; ++c) {
-      p = carry_ptr<D>(base, g, c, 0, n_chunks);
+      for (int e = 0; e < E; ++e) acc[e] = p[lane * E + e];
+      members = carry_cnt[((size_t)g * n_chunks + c0) * 2 + 1];
+      for (int cb = c0 + 1; cb <= c1; cb += 8) {
+        float x[8][E];
+        int m[8];
 #pragma unroll
-      for (int e = 0; e < E; ++e) { ak[e] += p[lane * E + e]; av[e] += p[D + lane * E + e]; }
-      members += carry_cnt[((size_t)g * n_chunks + c) * 2];
+        for (int u = 0; u < 8; ++u) {
+          const int c = min(cb + u, c1);
+          const float* pc = carry_ptr<D>(base, g, c, 0, n_chunks) + tensor * D;
+#pragma unroll
+          for (int e = 0; e < E; ++e) x[u][e] = pc[lane * E + e];
+          m[u] = carry_cnt[((size_t)g * n_chunks + c) * 2];
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (cb + u <= c1) {
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[e] += x[u][e];
+            members += m[u];
+          }
+        }
+      }
     }
-  }
-  const float c = (float)(members + 1);
-  store_row<T, E>(k_out + ((size_t)g * cap + slot) * D, lane, ak, c);
-  store_row<T, E>(v_out + ((size_t)g * cap + slot) * D, lane, av, c);
-  if (lane == 0) counts[(size_t)g * cap + slot] = members + 1;
+    store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)(members + 1));
+    if (tensor == 0 && lane == 0) counts[(size_t)g * cap + slot] = members + 1;
   }
 }
 

@@ -311,13 +311,13 @@ void launch_seg_kernels(meda_ctx* ctx, const void* k, const void* v, const int32
   const int max_slots = std::min(cap, n);
   if (!evict) {
     LaunchScope scope(ctx, MEDA_K_REDUCE, st);
-    seg_reduce_kernel<T, D><<<dim3((ctx->seg_chunks + kSegWarps - 1) / kSegWarps, c.n_kv_heads), kSegWarps * 32, 0, st>>>(
+    seg_reduce_kernel<T, D><<<dim3((ctx->seg_chunks + kSegWarps - 1) / kSegWarps, c.n_kv_heads, 2), kSegWarps * 32, 0, st>>>(
         static_cast<const T*>(k), static_cast<const T*>(v), keys, rows, idx_conserved, budget_row,
         static_cast<T*>(k_out), static_cast<T*>(v_out), counts, ctx->ws.seg_start, ctx->ws.seg_end, ctx->ws.carry,
         ctx->ws.carry_cnt, n, cap, ctx->seg_chunks);
   }
   LaunchScope scope(ctx, MEDA_K_REDUCE, st);
-  seg_finalize_kernel<T, D><<<dim3(std::min((max_slots + 7) / 8, ctx->sm_count * 8), c.n_kv_heads), 256, 0, st>>>(
+  seg_finalize_kernel<T, D><<<dim3(std::min((max_slots + 7) / 8, ctx->sm_count * 8), c.n_kv_heads, 2), 256, 0, st>>>(
       static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, budget_row, ctx->ws.seg_start,
       ctx->ws.seg_end, ctx->ws.carry, ctx->ws.carry_cnt, static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n,
       cap, ctx->seg_chunks, evict);

@@ -34,7 +34,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 struct StatsPolicy {
   struct Params {
     const uint8_t* modality;     // padded to a multiple of 128 with the value 2 (= no key)
-    float* partial;              // [chunks][Hq][w][4]
+    float* partial;              // [chunks * 2][Hq][w][4]: one partial per (key chunk, epilogue group)
     int n, hq, group, w, cols;   // cols = group * w query rows per KV group
     int row_blocks;              // ceil(cols / 256)
     int chunks, tiles_per_chunk, tiles_total;
@@ -42,7 +42,9 @@ struct StatsPolicy {
   };
   static constexpr int kABuffers = 1;
   static constexpr int kBStages = 4;
-  static constexpr uint32_t kExtraBytes = kUsEpilogueWarps * 128;     // one modality slice per epilogue warp
+  static constexpr int kEpilogueGroups = 2;      // this sweep is bound by its epilogue: two tiles at a time
+  static constexpr uint32_t kExtraBytes = kEpilogueGroups * kUsEpilogueWarps * 128;   // one modality slice per epilogue warp
+  static constexpr uint32_t kItemExtraBytes = 0;
 
   __device__ static bool active(const Params&) { return true; }
   __device__ static bool get_item(const Params& p, int it, StreamItem& o) {
@@ -65,20 +67,65 @@ struct StatsPolicy {
 
   struct Epilogue {
     uint8_t* mod_t;
-    int lane, row_in_block;
+    int lane, row_in_block, group;
     float mv, zv, mt, zt;        // running (max, sum) in base-2 logit units, visual and text keys
     __device__ void init(const Params&, unsigned char* extra, int ewarp, int lane_) {
       mod_t = extra + ewarp * 128;
       lane = lane_;
-      row_in_block = (ewarp / 4) * 128 + ((ewarp + 2) % 4) * 32 + lane_;
+      group = ewarp / kUsEpilogueWarps;
+      row_in_block = ((ewarp % kUsEpilogueWarps) / 4) * 128 + ((ewarp + 2) % 4) * 32 + lane_;
     }
-    __device__ void item_begin(const Params&, const StreamItem&) {
+    __device__ void item_begin(const Params&, const StreamItem&, const unsigned char*) {
       mv = mt = -INFINITY;
       zv = zt = 0.f;
     }
     __device__ __forceinline__ static void absorb(float& m, float& z, float t) {
       if (t > m) { z = z * fast_exp2(m - t) + 1.f; m = t; }
       else z += fast_exp2(t - m);
+    }
+    // 32 consecutive keys starting at j0 against this thread's query row.
+    __device__ __forceinline__ void chunk(const Params& p, const uint32_t (&r)[32], int chunk_idx, int j0,
+                                          int last_visible) {
+      const uint4 ma = reinterpret_cast<const uint4*>(mod_t + chunk_idx * 32)[0];
+      const uint4 mb = reinterpret_cast<const uint4*>(mod_t + chunk_idx * 32)[1];
+      const uint32_t all_or = ma.x | ma.y | ma.z | ma.w | mb.x | mb.y | mb.z | mb.w;
+      const uint32_t all_and = ma.x & ma.y & ma.z & ma.w & mb.x & mb.y & mb.z & mb.w;
+      const bool uniform_text = all_or == 0u;
+      const bool uniform_visual = all_and == 0x01010101u && all_or == 0x01010101u;
+      if ((uniform_text || uniform_visual) && j0 + 31 <= last_visible) {
+        // one modality, all keys visible: chunk maximum first (three-input maxima), then one exp2 per key
+        float t[12];
+#pragma unroll
+        for (int x = 0; x < 10; ++x)
+          t[x] = sm100::fmax3(__uint_as_float(r[3 * x]), __uint_as_float(r[3 * x + 1]), __uint_as_float(r[3 * x + 2]));
+        t[10] = __uint_as_float(r[30]);
+        t[11] = __uint_as_float(r[31]);
+        const float u0 = sm100::fmax3(t[0], t[1], t[2]), u1 = sm100::fmax3(t[3], t[4], t[5]);
+        const float u2 = sm100::fmax3(t[6], t[7], t[8]), u3 = sm100::fmax3(t[9], t[10], t[11]);
+        const float cm = fmaxf(sm100::fmax3(u0, u1, u2), u3);
+        float& m = uniform_visual ? mv : mt;
+        float& z = uniform_visual ? zv : zt;
+        const float m_new = fmaxf(m, cm * p.sc2);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int x = 0; x < 32; x += 4) {
+          a0 += fast_exp2(fmaf(__uint_as_float(r[x + 0]), p.sc2, -m_new));
+          a1 += fast_exp2(fmaf(__uint_as_float(r[x + 1]), p.sc2, -m_new));
+          a2 += fast_exp2(fmaf(__uint_as_float(r[x + 2]), p.sc2, -m_new));
+          a3 += fast_exp2(fmaf(__uint_as_float(r[x + 3]), p.sc2, -m_new));
+        }
+        z = z * fast_exp2(m - m_new) + ((a0 + a1) + (a2 + a3));
+        m = m_new;
+      } else {
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+          const int md = mod_t[chunk_idx * 32 + x];
+          if (md < 2 && j0 + x <= last_visible) {
+            if (md == MEDA_VISUAL) absorb(mv, zv, __uint_as_float(r[x]) * p.sc2);
+            else absorb(mt, zt, __uint_as_float(r[x]) * p.sc2);
+          }
+        }
+      }
     }
     __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
       const int rb = it.u0 & 65535;
@@ -91,43 +138,24 @@ struct StatsPolicy {
       reinterpret_cast<uint32_t*>(mod_t)[lane] = __ldg(reinterpret_cast<const uint32_t*>(p.modality + c0) + lane);
       __syncwarp();
       if (!__any_sync(0xffffffffu, valid)) return;
-#pragma unroll 1
-      for (int chunk = 0; chunk < 4; ++chunk) {
-        float v[32];
-        __syncwarp();
-        sm100::tmem_ld_32x32(taddr + chunk * 32u, v);
-        if (valid) {
-        const int j0 = c0 + chunk * 32;
-        const uint4 ma = reinterpret_cast<const uint4*>(mod_t + chunk * 32)[0];
-        const uint4 mb = reinterpret_cast<const uint4*>(mod_t + chunk * 32)[1];
-        const uint32_t all_or = ma.x | ma.y | ma.z | ma.w | mb.x | mb.y | mb.z | mb.w;
-        const uint32_t all_and = ma.x & ma.y & ma.z & ma.w & mb.x & mb.y & mb.z & mb.w;
-        const bool uniform_text = all_or == 0u;
-        const bool uniform_visual = all_and == 0x01010101u && all_or == 0x01010101u;
-        if ((uniform_text || uniform_visual) && j0 + 31 <= last_visible) {
-          float cm = v[0];
-#pragma unroll
-          for (int x = 1; x < 32; ++x) cm = fmaxf(cm, v[x]);
-          float& m = uniform_visual ? mv : mt;
-          float& z = uniform_visual ? zv : zt;
-          const float m_new = fmaxf(m, cm * p.sc2);
-          float acc = 0.f;
-#pragma unroll
-          for (int x = 0; x < 32; ++x) acc += fast_exp2(fmaf(v[x], p.sc2, -m_new));
-          z = z * fast_exp2(m - m_new) + acc;
-          m = m_new;
-        } else {
-#pragma unroll
-          for (int x = 0; x < 32; ++x) {
-            const int md = mod_t[chunk * 32 + x];
-            if (md < 2 && j0 + x <= last_visible) {
-              if (md == MEDA_VISUAL) absorb(mv, zv, v[x] * p.sc2);
-              else absorb(mt, zt, v[x] * p.sc2);
-            }
-          }
-        }
-        }
-      }
+      // two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced
+      uint32_t ra[32], rb2[32];
+      sm100::tmem_ld_32x32_issue(taddr, ra);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(ra);
+      sm100::tmem_ld_32x32_issue(taddr + 32u, rb2);
+      if (valid) chunk(p, ra, 0, c0, last_visible);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(rb2);
+      sm100::tmem_ld_32x32_issue(taddr + 64u, ra);
+      if (valid) chunk(p, rb2, 1, c0 + 32, last_visible);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(ra);
+      sm100::tmem_ld_32x32_issue(taddr + 96u, rb2);
+      if (valid) chunk(p, ra, 2, c0 + 64, last_visible);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(rb2);
+      if (valid) chunk(p, rb2, 3, c0 + 96, last_visible);
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {
       const int g = it.u0 >> 16, rb = it.u0 & 65535;
@@ -143,7 +171,7 @@ struct StatsPolicy {
       out.y = z_all;
       out.z = mv * kLn2;
       out.w = zv;
-      reinterpret_cast<float4*>(p.partial)[((size_t)it.u1 * p.hq + h) * p.w + i] = out;
+      reinterpret_cast<float4*>(p.partial)[((size_t)(it.u1 * kEpilogueGroups + group) * p.hq + h) * p.w + i] = out;
     }
   };
 };
@@ -172,9 +200,13 @@ __global__ void sweep_coef_kernel(const float* __restrict__ row_stats, float4* _
 }
 
 // ---------------------------------------------------------------------------------------------
-// Sweep 2: scores and entropy.  W = window (32 or 64).
+// Sweep 2: scores and entropy.  W = window (32 or 64), MODE = entropy_mode.  The per-column constants
+// of the item's KV group travel with the resident key block (bulk copies on the same barrier) and
+// are read from shared memory, one broadcast load per logit.
 // ---------------------------------------------------------------------------------------------
-template <int W>
+constexpr int kSweepMaxCols = 512;                     // query rows per KV group the tensor-core sweep accepts
+
+template <int W, int MODE>
 struct SweepPolicy {
   struct Params {
     const uint8_t* modality;     // padded as above
@@ -182,14 +214,16 @@ struct SweepPolicy {
     const float2* text;          // [Hq * w]
     float* scores;               // [Hkv][n] or null
     float* ent_partial;          // [blocks * 8] or null
-    int n, hkv, cols;            // cols = group * W columns per KV head
+    int n, hkv, cols;            // cols = group * W columns per KV head (multiple of 32, <= kSweepMaxCols)
     int n_blocks;                // ceil(n / 256)
-    int entropy_mode;
     float sc2;
   };
   static constexpr int kABuffers = 2;
   static constexpr int kBStages = 2;
+  static constexpr int kEpilogueGroups = 1;
   static constexpr uint32_t kExtraBytes = 0;
+  static constexpr uint32_t kTextOff = kSweepMaxCols * 16;
+  static constexpr uint32_t kItemExtraBytes = kSweepMaxCols * (16 + 8);
 
   __device__ static bool active(const Params&) { return true; }
   // Each block takes whole 256-key blocks and walks all KV heads of a block back to back, so that
@@ -209,11 +243,18 @@ struct SweepPolicy {
     o.u1 = blk;
     return true;
   }
+  __device__ static uint32_t item_extra_bytes(const Params& p, const StreamItem&) { return (uint32_t)p.cols * 24u; }
+  __device__ static void item_extra_issue(const Params& p, const StreamItem& it, unsigned char* dst, uint64_t* bar) {
+    sm100::bulk_load(dst, p.vis + it.b_row, (uint32_t)p.cols * 16u, bar);
+    sm100::bulk_load(dst + kTextOff, p.text + it.b_row, (uint32_t)p.cols * 8u, bar);
+  }
 
   struct Epilogue {
     int lane, ewarp, row_in_block;
+    const float4* cvis;          // this item's constants, shared memory
+    const float2* ctext;
     float abar[W];               // head-averaged visual-softmax attention of this key, per window row
-    float plogp;                 // entropy_mode 1 accumulator
+    float plogp;                 // MODE 1 accumulator
     float score;
     __device__ void init(const Params&, unsigned char*, int ewarp_, int lane_) {
       lane = lane_;
@@ -223,29 +264,51 @@ struct SweepPolicy {
       for (int x = 0; x < W; ++x) abar[x] = 0.f;
       plogp = 0.f;
     }
-    __device__ void item_begin(const Params&, const StreamItem&) { score = 0.f; }
+    __device__ void item_begin(const Params&, const StreamItem&, const unsigned char* item_extra) {
+      score = 0.f;
+      cvis = reinterpret_cast<const float4*>(item_extra);
+      ctext = reinterpret_cast<const float2*>(item_extra + kTextOff);
+    }
 
-    template <int OFF>
-    __device__ __forceinline__ void chunk_visual(const Params& p, const float (&v)[32], int col0, int first_row) {
+    // A visual key against 32 query columns (one head's window rows OFF .. OFF + 31).  MASK: the key
+    // lies inside the window, so rows before first_row do not see it.
+    template <int OFF, bool MASK>
+    __device__ __forceinline__ void chunk_visual(const Params& p, const uint32_t (&r)[32], const float4* c4, int first_row) {
 #pragma unroll
       for (int x = 0; x < 32; ++x) {
-        const float4 c = __ldg(p.vis + col0 + x);
-        const float t = fmaf(v[x], p.sc2, -c.x);
+        const float4 c = c4[x];
+        const float t = fmaf(__uint_as_float(r[x]), p.sc2, -c.x);
         float e = fast_exp2(t);
-        if (OFF + x < first_row) e = 0.f;
+        if (MASK && OFF + x < first_row) e = 0.f;
         score = fmaf(e, c.y, score);
-        const float pv = e * c.z;
-        if (p.entropy_mode == 0) abar[OFF + x] += pv;
-        else plogp = fmaf(pv, fmaf(t, kLn2, c.w), plogp);
+        if (MODE == 0) abar[OFF + x] = fmaf(e, c.z, abar[OFF + x]);
+        else plogp = fmaf(e * c.z, fmaf(t, kLn2, c.w), plogp);
       }
     }
-    __device__ __forceinline__ void chunk_text(const Params& p, const float (&v)[32], int col0, int row0, int first_row) {
+    template <bool MASK>
+    __device__ __forceinline__ void chunk_text(const Params& p, const uint32_t (&r)[32], const float2* c2, int row0, int first_row) {
 #pragma unroll
       for (int x = 0; x < 32; ++x) {
-        const float2 c = __ldg(p.text + col0 + x);
-        float e = fast_exp2(fmaf(v[x], p.sc2, -c.x));
-        if (row0 + x < first_row) e = 0.f;
+        const float2 c = c2[x];
+        float e = fast_exp2(fmaf(__uint_as_float(r[x]), p.sc2, -c.x));
+        if (MASK && row0 + x < first_row) e = 0.f;
         score = fmaf(e, c.y, score);
+      }
+    }
+    __device__ __forceinline__ void chunk(const Params& p, const uint32_t (&r)[32], int local, int md, int first_row,
+                                          bool masked) {
+      const int row0 = local % W;                       // local = column inside the KV group: head * W + row
+      if (md == MEDA_VISUAL) {
+        if (masked) {
+          if (W == 32 || row0 == 0) chunk_visual<0, true>(p, r, cvis + local, first_row);
+          else chunk_visual<(W > 32 ? 32 : 0), true>(p, r, cvis + local, first_row);
+        } else {
+          if (W == 32 || row0 == 0) chunk_visual<0, false>(p, r, cvis + local, first_row);
+          else chunk_visual<(W > 32 ? 32 : 0), false>(p, r, cvis + local, first_row);
+        }
+      } else {
+        if (masked) chunk_text<true>(p, r, ctext + local, row0, first_row);
+        else chunk_text<false>(p, r, ctext + local, row0, first_row);
       }
     }
     __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
@@ -253,23 +316,32 @@ struct SweepPolicy {
       const bool valid = j < p.n;
       const int md = p.modality[j];                        // the padded map covers j up to the block end
       const int first_row = j - (p.n - W);                 // causal: window rows i >= first_row see key j
+      const bool masked = __any_sync(0xffffffffu, valid && first_row > 0);
       const int n_chunks = (tile == it.n_tiles - 1 ? it.last_n : 128) / 32;
-#pragma unroll 1
-      for (int chunk = 0; chunk < n_chunks; ++chunk) {
-        float v[32];
-        __syncwarp();
-        sm100::tmem_ld_32x32(taddr + chunk * 32u, v);
-        if (valid) {
-          const int local = tile * 128 + chunk * 32;          // column inside the KV group: head * W + row
-          const int col0 = it.b_row + local;
-          const int row0 = local % W;
-          if (md == MEDA_VISUAL) {
-            if (W == 32 || row0 == 0) chunk_visual<0>(p, v, col0, first_row);
-            else chunk_visual<(W > 32 ? 32 : 0)>(p, v, col0, first_row);
-          } else {
-            chunk_text(p, v, col0, row0, first_row);
-          }
-        }
+      const int local0 = tile * 128;
+      // two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced
+      uint32_t ra[32], rb[32];
+      sm100::tmem_ld_32x32_issue(taddr, ra);
+      sm100::tmem_ld_wait();
+      sm100::tmem_ld_pin(ra);
+      if (n_chunks > 1) sm100::tmem_ld_32x32_issue(taddr + 32u, rb);
+      if (valid) chunk(p, ra, local0, md, first_row, masked);
+      if (n_chunks > 1) {
+        sm100::tmem_ld_wait();
+        sm100::tmem_ld_pin(rb);
+        if (n_chunks > 2) sm100::tmem_ld_32x32_issue(taddr + 64u, ra);
+        if (valid) chunk(p, rb, local0 + 32, md, first_row, masked);
+      }
+      if (n_chunks > 2) {
+        sm100::tmem_ld_wait();
+        sm100::tmem_ld_pin(ra);
+        if (n_chunks > 3) sm100::tmem_ld_32x32_issue(taddr + 96u, rb);
+        if (valid) chunk(p, ra, local0 + 64, md, first_row, masked);
+      }
+      if (n_chunks > 3) {
+        sm100::tmem_ld_wait();
+        sm100::tmem_ld_pin(rb);
+        if (valid) chunk(p, rb, local0 + 96, md, first_row, masked);
       }
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {
@@ -278,7 +350,7 @@ struct SweepPolicy {
       if (it.u0 == p.hkv - 1) {
         // all heads of this key block are in: entropy partial of this warp's 32 keys
         float acc = plogp;
-        if (p.entropy_mode == 0) {
+        if (MODE == 0) {
 #pragma unroll
           for (int x = 0; x < W; ++x) {
             const float a = abar[x];

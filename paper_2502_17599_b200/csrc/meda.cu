@@ -212,22 +212,24 @@ meda_status launch_stats_fast(meda_ctx* ctx, const void* q_win, const void* k, f
   const int items = c.n_kv_heads * prm.row_blocks * prm.chunks;
   {
     LaunchScope scope(ctx, MEDA_K_STATS, st);
-    umma_stream_kernel<StatsPolicy><<<std::min(items, ctx->sm_count), kUsThreads, StreamShared<StatsPolicy>::alloc, st>>>(
+    umma_stream_kernel<StatsPolicy><<<std::min(items, ctx->sm_count), us_threads<StatsPolicy>(), StreamShared<StatsPolicy>::alloc, st>>>(
         map_q, map_k, prm, ctx->ws.status);
   }
   {
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
-    stats_combine_kernel<<<(c.n_q_heads * c.window + 7) / 8, 256, 0, st>>>(ctx->ws.stats_partial, row_stats, prm.chunks,
+    stats_combine_kernel<<<(c.n_q_heads * c.window + 7) / 8, 256, 0, st>>>(ctx->ws.stats_partial, row_stats,
+                                                                               prm.chunks * StatsPolicy::kEpilogueGroups,
                                                                                c.n_q_heads * c.window);
   }
   return launch_status();
 }
 
-template <int W>
+template <int W, int MODE>
 void launch_sweep_policy(meda_ctx* ctx, const CUtensorMap& map_k, const CUtensorMap& map_q, float* scores,
                          bool want_entropy, cudaStream_t st) {
   const meda_config& c = ctx->cfg;
-  typename SweepPolicy<W>::Params prm;
+  using Policy = SweepPolicy<W, MODE>;
+  typename Policy::Params prm;
   prm.modality = ctx->ws.modality;
   prm.vis = ctx->ws.coef_vis;
   prm.text = ctx->ws.coef_text;
@@ -235,10 +237,15 @@ void launch_sweep_policy(meda_ctx* ctx, const CUtensorMap& map_k, const CUtensor
   prm.ent_partial = want_entropy ? ctx->ws.ent_partial : nullptr;
   prm.n = c.n_tokens; prm.hkv = c.n_kv_heads; prm.cols = ctx->group * c.window;
   prm.n_blocks = (c.n_tokens + 255) / 256;
-  prm.entropy_mode = c.entropy_mode;
   prm.sc2 = kLog2e / sqrtf((float)c.head_dim);
-  umma_stream_kernel<SweepPolicy<W>><<<std::min(prm.n_blocks, ctx->sm_count), kUsThreads, StreamShared<SweepPolicy<W>>::alloc, st>>>(
+  umma_stream_kernel<Policy><<<std::min(prm.n_blocks, ctx->sm_count), us_threads<Policy>(), StreamShared<Policy>::alloc, st>>>(
       map_k, map_q, prm, ctx->ws.status);
+}
+
+template <int W, int MODE>
+meda_status raise_sweep_smem() {
+  return cudaFuncSetAttribute(umma_stream_kernel<SweepPolicy<W, MODE>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)StreamShared<SweepPolicy<W, MODE>>::alloc) == cudaSuccess ? MEDA_OK : MEDA_ERR_CUDA;
 }
 
 meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
@@ -257,8 +264,11 @@ meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, c
   }
   {
     LaunchScope scope(ctx, MEDA_K_SWEEP, st);
-    if (c.window == 32) launch_sweep_policy<32>(ctx, map_k, map_q, scores, entropy != nullptr, st);
-    else launch_sweep_policy<64>(ctx, map_k, map_q, scores, entropy != nullptr, st);
+    const bool e = entropy != nullptr;
+    if (c.window == 32 && c.entropy_mode == 0) launch_sweep_policy<32, 0>(ctx, map_k, map_q, scores, e, st);
+    else if (c.window == 32) launch_sweep_policy<32, 1>(ctx, map_k, map_q, scores, e, st);
+    else if (c.entropy_mode == 0) launch_sweep_policy<64, 0>(ctx, map_k, map_q, scores, e, st);
+    else launch_sweep_policy<64, 1>(ctx, map_k, map_q, scores, e, st);
   }
   if (entropy) {
     LaunchScope scope(ctx, MEDA_K_ENTROPY_FINAL, st);
@@ -290,7 +300,7 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
     const int items = ((n + 255) / 256) * c.n_kv_heads;
     NearestPolicy::Params prm{ctx->ws.inv_norm, budget_row, ctx->ws.token_target, n, c.n_kv_heads, cap, ctx->inv_stride};
     LaunchScope scope(ctx, MEDA_K_NEAREST, st);
-    umma_stream_kernel<NearestPolicy><<<std::min(items, ctx->sm_count), kUsThreads, StreamShared<NearestPolicy>::alloc, st>>>(
+    umma_stream_kernel<NearestPolicy><<<std::min(items, ctx->sm_count), us_threads<NearestPolicy>(), StreamShared<NearestPolicy>::alloc, st>>>(
         map_k, map_kc, prm, ctx->ws.status);
   }
   {
@@ -535,7 +545,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     return MEDA_ERR_CUDA;
   }
   ctx->fast = c.dtype == MEDA_BF16 && c.head_dim == kFastDim;
-  ctx->fast_attn = ctx->fast && (c.window == 32 || c.window == 64);
+  ctx->fast_attn = ctx->fast && (c.window == 32 || c.window == 64) && ctx->group * c.window <= kSweepMaxCols;
   ctx->ent_slots = std::max(generic_tiles(c.n_tokens), ((c.n_tokens + 255) / 256) * kUsEpilogueWarps);
   {
     // key chunks of the tensor-core normaliser sweep: about two items per SM
@@ -555,16 +565,16 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   if (st == MEDA_OK && cudaMemset(ws.modality, 2, (size_t)mod_bytes) != cudaSuccess) st = MEDA_ERR_CUDA;
   if (st == MEDA_OK) st = carve(&ws.status, 1, &ws.bytes);
   if (st == MEDA_OK)
-    st = carve(&ws.stats_partial, (int64_t)std::max(kStatsChunks, ctx->stats_chunks) * c.n_q_heads * c.window * 4, &ws.bytes);
+    st = carve(&ws.stats_partial, (int64_t)std::max(kStatsChunks, ctx->stats_chunks * StatsPolicy::kEpilogueGroups) * c.n_q_heads * c.window * 4, &ws.bytes);
   if (ctx->fast_attn) {
     if (st == MEDA_OK) st = carve(&ws.coef_vis, (int64_t)c.n_q_heads * c.window, &ws.bytes);
     if (st == MEDA_OK) st = carve(&ws.coef_text, (int64_t)c.n_q_heads * c.window, &ws.bytes);
     if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<StatsPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)StreamShared<StatsPolicy>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
-    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<SweepPolicy<32>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)StreamShared<SweepPolicy<32>>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
-    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<SweepPolicy<64>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)StreamShared<SweepPolicy<64>>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK) st = raise_sweep_smem<32, 0>();
+    if (st == MEDA_OK) st = raise_sweep_smem<32, 1>();
+    if (st == MEDA_OK) st = raise_sweep_smem<64, 0>();
+    if (st == MEDA_OK) st = raise_sweep_smem<64, 1>();
   }
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
   ctx->sort_chunks = (int)((n + kSortBlockItems - 1) / kSortBlockItems + 7) / 8 * 8;   // padded: the scan works on whole vectors

@@ -63,6 +63,8 @@ struct NearestPolicy {
   static constexpr int kABuffers = 1;
   static constexpr int kBStages = 4;
   static constexpr uint32_t kExtraBytes = kUsEpilogueWarps * 128 * 4;   // one inverse-norm slice per epilogue warp
+  static constexpr uint32_t kItemExtraBytes = 0;
+  static constexpr int kEpilogueGroups = 1;
 
   __device__ static int slots(const Params& p) { return min(p.budget_row[0], p.cap); }
   __device__ static bool active(const Params& p) {
@@ -101,7 +103,7 @@ struct NearestPolicy {
       lane = lane_;
       row_in_block = (ewarp / 4) * 128 + ((ewarp + 2) % 4) * 32 + lane_;   // (ewarp + 2) % 4 == warp % 4
     }
-    __device__ void item_begin(const Params&, const StreamItem&) {
+    __device__ void item_begin(const Params&, const StreamItem&, const unsigned char*) {
       best = -INFINITY;
       best_slot = 0;
     }

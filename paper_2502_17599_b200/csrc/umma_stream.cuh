@@ -8,18 +8,27 @@
 //   warp 0      : TMA producer (one elected lane)
 //   warp 1      : tensor-memory owner and UMMA issuer (one elected lane)
 //   warps 2..9  : epilogue; warp e reads the 32 TMEM lanes (warp % 4) * 32.. of UMMA tile (e / 4)
+//   warps 10..17: (policies with kEpilogueGroups = 2) a second epilogue group with the same lane map.
+//                 Group g then reduces accumulator buffer g, i.e. every other streamed tile, so two
+//                 tiles are in the epilogue at any time; the policy combines what the two groups hold.
 //
 // What an item is and what the epilogue does with the accumulators is supplied by a policy type:
 //
 //   struct Policy {
 //     struct Params;                                  // trivially copyable kernel argument
 //     static constexpr int kABuffers, kBStages;       // resident-block buffers (1 or 2), B ring depth
+//     static constexpr int kEpilogueGroups;           // 1 or 2 groups of eight epilogue warps
 //     static constexpr uint32_t kExtraBytes;          // policy-owned shared memory
+//     static constexpr uint32_t kItemExtraBytes;      // per-item side data (multiple of 128), or 0; when
+//                                                     // non-zero it is bulk-copied next to the resident
+//                                                     // block, one copy per A buffer, and released with it:
+//     static uint32_t item_extra_bytes(const Params&, const StreamItem&);              // bytes of this item
+//     static void item_extra_issue(const Params&, const StreamItem&, unsigned char* dst, uint64_t* bar);
 //     static bool active(const Params&);              // false: the whole grid returns at once
 //     static bool get_item(const Params&, int it, StreamItem&);   // it-th item of this block, or false
 //     struct Epilogue {                               // one object per epilogue thread
-//       void init(const Params&, unsigned char* extra, int ewarp, int lane);
-//       void item_begin(const Params&, const StreamItem&);
+//       void init(const Params&, unsigned char* extra, int ewarp, int lane);   // ewarp 0..8 * groups - 1
+//       void item_begin(const Params&, const StreamItem&, const unsigned char* item_extra);
 //       void tile(const Params&, const StreamItem&, int tile, uint32_t taddr);   // taddr: this warp's lanes
 //       void item_end(const Params&, const StreamItem&);
 //     };
@@ -35,8 +44,9 @@
 namespace meda {
 
 constexpr int kFastDim = 128;                         // head_dim of the tensor-core paths
-constexpr int kUsThreads = 320;
-constexpr int kUsEpilogueWarps = 8;
+constexpr int kUsEpilogueWarps = 8;                   // per epilogue group
+template <class P>
+constexpr int us_threads() { return 64 + 32 * kUsEpilogueWarps * P::kEpilogueGroups; }
 constexpr uint32_t kUsHalfTile = 128 * 64 * 2;        // one 128-row x 64-column bf16 TMA box (16 KB)
 constexpr uint32_t kUsABlock = 4 * kUsHalfTile;       // 2 UMMA tiles x 2 K halves
 constexpr uint32_t kUsBStage = 2 * kUsHalfTile;       // 1 tile x 2 K halves
@@ -56,7 +66,8 @@ struct StreamShared {
   static constexpr uint32_t a_off = 0;
   static constexpr uint32_t b_off = a_off + P::kABuffers * kUsABlock;
   static constexpr uint32_t extra_off = b_off + P::kBStages * kUsBStage;
-  static constexpr uint32_t bar_off = extra_off + ((P::kExtraBytes + 15u) / 16u) * 16u;
+  static constexpr uint32_t item_extra_off = extra_off + ((P::kExtraBytes + 127u) / 128u) * 128u;
+  static constexpr uint32_t bar_off = item_extra_off + P::kABuffers * P::kItemExtraBytes;
   static constexpr uint32_t n_bars = 2 * P::kABuffers + 2 * P::kBStages + 4;
   static constexpr uint32_t misc_off = bar_off + n_bars * 8;
   static constexpr uint32_t total = misc_off + 16;
@@ -64,17 +75,20 @@ struct StreamShared {
 };
 
 template <class P>
-__global__ void __launch_bounds__(kUsThreads, 1)
+__global__ void __launch_bounds__(us_threads<P>(), 1)
 umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const typename P::Params prm, int* status) {
   using namespace sm100;
   using SH = StreamShared<P>;
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem =
-      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // aligned to 1024 bytes by pointer arithmetic on the shared array, so that every pointer derived from
+  // it is still known to point into shared memory
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* a_smem = smem + SH::a_off;
   unsigned char* b_smem = smem + SH::b_off;
   unsigned char* extra = smem + SH::extra_off;
+  unsigned char* item_extra = smem + SH::item_extra_off;
+  constexpr bool kHasItemExtra = P::kItemExtraBytes > 0;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SH::bar_off);
   uint64_t* a_full = bars;
   uint64_t* a_empty = a_full + P::kABuffers;
@@ -89,7 +103,11 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < P::kABuffers; ++i) { mbar_init(a_full + i, 1); mbar_init(a_empty + i, 1); }
+    // with per-item side data the epilogue warps read the A buffer's slot too and release it with the UMMAs
+    for (int i = 0; i < P::kABuffers; ++i) {
+      mbar_init(a_full + i, 1);
+      mbar_init(a_empty + i, kHasItemExtra ? 1 + kUsEpilogueWarps * P::kEpilogueGroups : 1);
+    }
     for (int s = 0; s < P::kBStages; ++s) { mbar_init(b_full + s, 1); mbar_init(b_empty + s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(t_full + b, 1); mbar_init(t_empty + b, kUsEpilogueWarps); }
     *abort_flag = 0;
@@ -116,11 +134,15 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         const uint32_t abuf = (uint32_t)i % P::kABuffers, aphase = ((uint32_t)i / P::kABuffers) & 1u;
         ok = mbar_wait(a_empty + abuf, aphase ^ 1u, abort_flag);
         if (!ok) break;
-        mbar_expect_tx(a_full + abuf, 2 * kUsHalfTile * it.m_tiles);
+        uint32_t side_bytes = 0;
+        if constexpr (kHasItemExtra) side_bytes = P::item_extra_bytes(prm, it);
+        mbar_expect_tx(a_full + abuf, 2 * kUsHalfTile * it.m_tiles + side_bytes);
         for (int t = 0; t < it.m_tiles; ++t)
           for (int kh = 0; kh < 2; ++kh)
             tma_load_3d(a_smem + abuf * kUsABlock + (t * 2 + kh) * kUsHalfTile, &map_a, a_full + abuf, kh * 64,
                         it.a_row + t * 128, it.a_head);
+        if constexpr (kHasItemExtra)
+          P::item_extra_issue(prm, it, item_extra + abuf * P::kItemExtraBytes, a_full + abuf);
         for (int tile = 0; tile < it.n_tiles; ++tile, ++b_count) {
           const uint32_t stage = b_count % P::kBStages, phase = (b_count / P::kBStages) & 1u;
           ok = mbar_wait(b_empty + stage, phase ^ 1u, abort_flag);
@@ -170,17 +192,25 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   } else {
     // ------------------------------------------------------------------ epilogue
     const int ewarp = warp - 2;
+    const int group = ewarp / kUsEpilogueWarps;
     const int quarter = warp % 4;                 // TMEM lanes this warp may read: 32 * (warp % 4) ..
-    const int t = ewarp / 4;                      // which UMMA tile of the resident block
+    const int t = (ewarp % kUsEpilogueWarps) / 4; // which UMMA tile of the resident block
     typename P::Epilogue ep;
     ep.init(prm, extra, ewarp, lane);
     uint32_t t_count = 0;
     StreamItem it;
     bool ok = true;
     for (int i = 0; ok && P::get_item(prm, i, it); ++i) {
-      ep.item_begin(prm, it);
+      const uint32_t abuf = (uint32_t)i % P::kABuffers, aphase = ((uint32_t)i / P::kABuffers) & 1u;
+      if constexpr (kHasItemExtra) {
+        ok = mbar_wait(a_full + abuf, aphase, abort_flag);          // the side data has landed
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+      ep.item_begin(prm, it, item_extra + abuf * P::kItemExtraBytes);
       for (int tile = 0; tile < it.n_tiles; ++tile, ++t_count) {
         const uint32_t buf = t_count & 1u, tphase = (t_count >> 1) & 1u;
+        if (P::kEpilogueGroups == 2 && (int)buf != group) continue;   // the other group's tile
         ok = mbar_wait(t_full + buf, tphase, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -192,6 +222,10 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (lane == 0) mbar_arrive(t_empty + buf);
       }
       if (ok) ep.item_end(prm, it);
+      if constexpr (kHasItemExtra) {
+        __syncwarp();
+        if (ok && lane == 0) mbar_arrive(a_empty + abuf);          // this warp no longer reads the side data
+      }
     }
   }
 

@@ -270,45 +270,42 @@ struct SweepPolicy {
       ctext = reinterpret_cast<const float2*>(item_extra + kTextOff);
     }
 
-    // A visual key against 32 query columns (one head's window rows OFF .. OFF + 31).  MASK: the key
-    // lies inside the window, so rows before first_row do not see it.
-    template <int OFF, bool MASK>
-    __device__ __forceinline__ void chunk_visual(const Params& p, const uint32_t (&r)[32], const float4* c4, int first_row) {
+    // A visual key against 32 query columns (one head's window rows OFF .. OFF + 31), all of which see it.
+    template <int OFF>
+    __device__ __forceinline__ void chunk_visual(const Params& p, const uint32_t (&r)[32], const float4* c4) {
 #pragma unroll
       for (int x = 0; x < 32; ++x) {
         const float4 c = c4[x];
         const float t = fmaf(__uint_as_float(r[x]), p.sc2, -c.x);
-        float e = fast_exp2(t);
-        if (MASK && OFF + x < first_row) e = 0.f;
+        const float e = fast_exp2(t);
         score = fmaf(e, c.y, score);
         if (MODE == 0) abar[OFF + x] = fmaf(e, c.z, abar[OFF + x]);
         else plogp = fmaf(e * c.z, fmaf(t, kLn2, c.w), plogp);
       }
     }
-    template <bool MASK>
-    __device__ __forceinline__ void chunk_text(const Params& p, const uint32_t (&r)[32], const float2* c2, int row0, int first_row) {
+    __device__ __forceinline__ void chunk_text(const Params& p, const uint32_t (&r)[32], const float2* c2) {
 #pragma unroll
       for (int x = 0; x < 32; ++x) {
         const float2 c = c2[x];
-        float e = fast_exp2(fmaf(__uint_as_float(r[x]), p.sc2, -c.x));
-        if (MASK && row0 + x < first_row) e = 0.f;
-        score = fmaf(e, c.y, score);
+        score = fmaf(fast_exp2(fmaf(__uint_as_float(r[x]), p.sc2, -c.x)), c.y, score);
       }
     }
-    __device__ __forceinline__ void chunk(const Params& p, const uint32_t (&r)[32], int local, int md, int first_row,
+    // `masked`: some key of the warp lies inside the observation window (the last W of the sequence), so
+    // window rows before first_row do not see it.  Those logits are replaced by a hugely negative
+    // value, whose exp2 is exactly zero, and the ordinary routines run.  Only the last key block
+    // gets here.
+    __device__ __forceinline__ void chunk(const Params& p, uint32_t (&r)[32], int local, int md, int first_row,
                                           bool masked) {
-      const int row0 = local % W;                       // local = column inside the KV group: head * W + row
+      if (masked) {
+        const int row0 = local % W;
+#pragma unroll
+        for (int x = 0; x < 32; ++x) if (row0 + x < first_row) r[x] = __float_as_uint(-1e30f);
+      }
       if (md == MEDA_VISUAL) {
-        if (masked) {
-          if (W == 32 || row0 == 0) chunk_visual<0, true>(p, r, cvis + local, first_row);
-          else chunk_visual<(W > 32 ? 32 : 0), true>(p, r, cvis + local, first_row);
-        } else {
-          if (W == 32 || row0 == 0) chunk_visual<0, false>(p, r, cvis + local, first_row);
-          else chunk_visual<(W > 32 ? 32 : 0), false>(p, r, cvis + local, first_row);
-        }
+        if (W == 32 || local % W == 0) chunk_visual<0>(p, r, cvis + local);
+        else chunk_visual<(W > 32 ? 32 : 0)>(p, r, cvis + local);
       } else {
-        if (masked) chunk_text<true>(p, r, ctext + local, row0, first_row);
-        else chunk_text<false>(p, r, ctext + local, row0, first_row);
+        chunk_text(p, r, ctext + local);
       }
     }
     __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {

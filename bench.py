@@ -203,6 +203,32 @@ def algorithmic_work(wl, budgets):
     return out
 
 
+def rank_workload(name, rank, layers=0):
+    """The prompt rank `rank` compresses: the named workload with its own seed (independent prompts, so
+    N ranks do N times the work: weak scaling, no data-path collective)."""
+    from paper_2502_17599_b200 import workloads as W
+    wl = W.WORKLOADS[name]
+    wl = wl.with_(seed=wl.seed + 1000 * rank)
+    if layers > 0:
+        wl = wl.with_(name=f"{wl.name}_first{layers}layers", n_layers=min(layers, wl.n_layers))
+    return wl
+
+
+def max_over_ranks(ms, world, device):
+    """The slowest rank's time: the only value exchanged between ranks."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+def whole_job_throughput(wl, world, ms_step):
+    """token*layers per second over all ranks."""
+    return world * wl.n_layers * wl.n_tokens / (ms_step * 1e-3)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -221,9 +247,7 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
 
-    wl = W.WORKLOADS[args.workload].with_(seed=W.WORKLOADS[args.workload].seed + 1000 * rank)
-    if args.layers > 0:
-        wl = wl.with_(name=f"{wl.name}_first{args.layers}layers", n_layers=min(args.layers, wl.n_layers))
+    wl = rank_workload(args.workload, rank, args.layers)
     L = wl.n_layers
     qs, ks, vs = [], [], []
     for l in range(L):
@@ -262,11 +286,8 @@ def run_ours(args):
     prof = cp.ctx.profile_read()
     cp.ctx.profile_enable(False)
     cp.ctx.check()
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t[0]) / args.steps
-    value = world * L * wl.n_tokens / (ms_step * 1e-3)
+    ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
+    value = whole_job_throughput(wl, world, ms_step)
 
     # end-to-end leg: pinned host inputs -> device -> pass -> compacted caches back to the host
     e2e = None
@@ -287,11 +308,9 @@ def run_ours(args):
         barrier()
         wall = (time.perf_counter() - t0) * 1e3
         ms_e2e = max(e0.elapsed_time(e1), wall) / args.e2e_steps
-        te = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * L * wl.n_tokens / (float(te[0]) * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": float(te[0])}
+        ms_e2e = max_over_ranks(ms_e2e, world, "cuda")
+        e2e = {"value": whole_job_throughput(wl, world, ms_e2e), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e}
         del q_h, k_h, v_h, out_host
 
     if rank != 0:

@@ -16,6 +16,7 @@
 #include "group_reduce.cuh"
 #include "merge_generic.cuh"
 #include "nearest_sm100.cuh"
+#include "nearest_ts_sm100.cuh"
 #include "select.cuh"
 
 using namespace meda;
@@ -285,10 +286,8 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
   const meda_config& c = ctx->cfg;
   const int n = c.n_tokens;
   if ((reinterpret_cast<uintptr_t>(k) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
-  CUtensorMap map_k, map_kc;
-  if (!make_rows_map(ctx, &map_k, k, n, c.n_kv_heads, n, 128) ||
-      !make_rows_map(ctx, &map_kc, ctx->ws.kc, ctx->kc_rows, c.n_kv_heads, ctx->kc_rows, 128))
-    return MEDA_ERR_CUDA;
+  CUtensorMap map_kc;
+  if (!make_rows_map(ctx, &map_kc, ctx->ws.kc, ctx->kc_rows, c.n_kv_heads, ctx->kc_rows, kNtTileN)) return MEDA_ERR_CUDA;
   const int max_slots = std::min(cap, n);
   {
     LaunchScope scope(ctx, MEDA_K_PREP, st);
@@ -298,10 +297,10 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
   }
   {
     const int items = ((n + 255) / 256) * c.n_kv_heads;
-    NearestPolicy::Params prm{ctx->ws.inv_norm, budget_row, ctx->ws.token_target, n, c.n_kv_heads, cap, ctx->inv_stride};
+    NearestParams prm{static_cast<const __nv_bfloat16*>(k), ctx->ws.inv_norm, budget_row, ctx->ws.token_target,
+                      n, c.n_kv_heads, cap, ctx->inv_stride};
     LaunchScope scope(ctx, MEDA_K_NEAREST, st);
-    umma_stream_kernel<NearestPolicy><<<std::min(items, ctx->sm_count), us_threads<NearestPolicy>(), StreamShared<NearestPolicy>::alloc, st>>>(
-        map_k, map_kc, prm, ctx->ws.status);
+    nearest_kernel<<<std::min(items, ctx->sm_count), kNtThreads, NearestSmem::alloc, st>>>(map_kc, prm, ctx->ws.status);
   }
   {
     LaunchScope scope(ctx, MEDA_K_GROUP, st);
@@ -601,8 +600,8 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
       ctx->encode_tiled = resolve_encode_tiled();
       if (!ctx->encode_tiled) st = MEDA_ERR_CUDA;
     }
-    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<NearestPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)StreamShared<NearestPolicy>::alloc) != cudaSuccess)
+    if (st == MEDA_OK && cudaFuncSetAttribute(nearest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)NearestSmem::alloc) != cudaSuccess)
       st = MEDA_ERR_CUDA;
   }
   if (st == MEDA_OK) st = carve(&ws.target, hkv * n, &ws.bytes);

@@ -164,23 +164,24 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         const uint32_t abuf = (uint32_t)i % P::kABuffers, aphase = ((uint32_t)i / P::kABuffers) & 1u;
         ok = mbar_wait(a_full + abuf, aphase, abort_flag);
         if (!ok) break;
-        const uint32_t a_addr = smem_u32(a_smem + abuf * kUsABlock);
+        const uint32_t a_lo = umma_desc_lo_sw128(smem_u32(a_smem + abuf * kUsABlock));
         for (int tile = 0; tile < it.n_tiles; ++tile, ++b_count, ++t_count) {
           const uint32_t stage = b_count % P::kBStages, phase = (b_count / P::kBStages) & 1u;
           const uint32_t buf = t_count & 1u, tphase = (t_count >> 1) & 1u;
           ok = mbar_wait(b_full + stage, phase, abort_flag) && mbar_wait(t_empty + buf, tphase ^ 1u, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t b_addr = smem_u32(b_smem + stage * kUsBStage);
+          const uint32_t b_lo = umma_desc_lo_sw128(smem_u32(b_smem + stage * kUsBStage));
           const uint32_t idesc = umma_idesc_bf16(128, tile == it.n_tiles - 1 ? it.last_n : 128);
           for (int t = 0; t < it.m_tiles; ++t) {
             const uint32_t d_tmem = tmem_base + buf * 256u + t * 128u;
+            const uint32_t at_lo = a_lo + (uint32_t)t * ((2 * kUsHalfTile) >> 4);
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t kh = kk / 4, koff = (kk % 4) * 32;
-              const uint64_t da = umma_desc_k_sw128(a_addr + (t * 2 + kh) * kUsHalfTile, koff);
-              const uint64_t db = umma_desc_k_sw128(b_addr + kh * kUsHalfTile, koff);
-              umma_bf16(d_tmem, da, db, idesc, kk > 0 ? 1u : 0u);
+              // K slice kk: half kk / 4 of the tile, 32-byte step (kk % 4) inside the 128-byte swizzled row
+              constexpr uint32_t kHalfStep = kUsHalfTile >> 4;
+              const uint32_t off = (uint32_t)(kk / 4) * kHalfStep + (uint32_t)(kk % 4) * 2u;
+              umma_bf16_lohi(d_tmem, at_lo + off, b_lo + off, idesc, kk > 0 ? 1u : 0u);
             }
           }
           umma_commit(b_empty + stage);     // the B stage may be refilled once these UMMAs have read it

@@ -16,7 +16,6 @@
 #include "group_reduce.cuh"
 #include "merge_generic.cuh"
 #include "nearest_sm100.cuh"
-#include "nearest_ts_sm100.cuh"
 #include "select.cuh"
 
 using namespace meda;
@@ -53,7 +52,6 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.target);
   cudaFree(ws.idx_less);
   cudaFree(ws.kc);
-  cudaFree(ws.token_target);
   cudaFree(ws.coef_vis);
   cudaFree(ws.coef_text);
   for (int i = 0; i < 2; ++i) { cudaFree(ws.sort_keys[i]); cudaFree(ws.sort_rows[i]); }
@@ -297,15 +295,10 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
   }
   {
     const int items = ((n + 255) / 256) * c.n_kv_heads;
-    NearestParams prm{static_cast<const __nv_bfloat16*>(k), ctx->ws.inv_norm, budget_row, ctx->ws.token_target,
+    NearestParams prm{static_cast<const __nv_bfloat16*>(k), ctx->ws.inv_norm, budget_row, idx_less, target,
                       n, c.n_kv_heads, cap, ctx->inv_stride};
     LaunchScope scope(ctx, MEDA_K_NEAREST, st);
     nearest_kernel<<<std::min(items, ctx->sm_count), kNtThreads, NearestSmem::alloc, st>>>(map_kc, prm, ctx->ws.status);
-  }
-  {
-    LaunchScope scope(ctx, MEDA_K_GROUP, st);
-    remap_targets_kernel<<<dim3((n + 255) / 256, c.n_kv_heads), 256, 0, st>>>(ctx->ws.token_target, idx_less,
-                                                                              budget_row, target, n, cap);
   }
   return launch_status();
 }
@@ -593,7 +586,6 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   if (st == MEDA_OK) st = carve(&ws.inv_norm, hkv * ctx->inv_stride, &ws.bytes);
   if (ctx->fast) {
     if (st == MEDA_OK) st = carve(&ws.kc, hkv * ctx->kc_rows * kFastDim, &ws.bytes);
-    if (st == MEDA_OK) st = carve(&ws.token_target, hkv * n, &ws.bytes);
     if (st == MEDA_OK && cudaMemset(ws.kc, 0, (size_t)(hkv * ctx->kc_rows * kFastDim * 2)) != cudaSuccess) st = MEDA_ERR_CUDA;
     if (st == MEDA_OK && cudaMemset(ws.inv_norm, 0, (size_t)(hkv * ctx->inv_stride * 4)) != cudaSuccess) st = MEDA_ERR_CUDA;
     if (st == MEDA_OK) {

@@ -25,7 +25,6 @@ struct Workspace {
   float* ent_partial = nullptr;       // [ent_slots]
   float* inv_norm = nullptr;          // [Hkv][inv_stride]  1 / max(|k_c|, eps) per conserved slot
   __nv_bfloat16* kc = nullptr;        // [Hkv][kc_rows][128] gathered conserved keys (bf16, head_dim 128 only)
-  int32_t* token_target = nullptr;    // [Hkv][n] nearest slot of every token row (tensor-core path)
   int32_t* sort_keys[2] = {nullptr, nullptr};   // [Hkv][n] ping-pong: target slot of each sorted entry
   int32_t* sort_rows[2] = {nullptr, nullptr};   // [Hkv][n] ping-pong: token row of each sorted entry
   int32_t* sort_table = nullptr;      // [Hkv][bins][sort blocks] digit counts, then offsets

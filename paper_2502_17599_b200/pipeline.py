@@ -48,6 +48,25 @@ class CompressionPass:
             c.compress_layer(l, k_layers[l], v_layers[l], self.scores[l], self.budgets, self.k_out[l], self.v_out[l],
                              self.counts[l], self.idx_c[l], self.cap, stream)
 
+    def capture(self, q_layers, k_layers, v_layers):
+        """Records the whole pass (every launch of `run` on these buffers) into a CUDA graph, after one
+        ordinary run that loads the kernels.  `replay()` then enqueues the pass with a single graph
+        launch: no per-kernel launch cost on the host and shorter gaps between kernels on the device.
+        Returns the number of kernels in the graph."""
+        self.run(q_layers, k_layers, v_layers)
+        torch.cuda.synchronize()
+        before = self.ctx.launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(q_layers, k_layers, v_layers)
+        self.graph = graph
+        self.graph_kernels = self.ctx.launch_count() - before
+        return self.graph_kernels
+
+    def replay(self):
+        """Enqueues the captured pass on torch's current stream."""
+        self.graph.replay()
+
     def run_from_host(self, q_host, k_host, v_host, staging, out_host):
         """End-to-end variant: per-layer inputs in pinned HOST memory are copied to the device
         staging buffers, the pass runs, and the budgets plus the compacted caches (only the S_l live

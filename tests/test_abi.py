@@ -81,3 +81,25 @@ def test_product_path_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in text and "from oracle" not in text, f
+
+
+def test_tensor_core_kernels_keep_tensor_memory_loads_out_of_local_memory():
+    """The arg-max kernel keeps a tcgen05.ld in flight while it works on the previous registers.  If the
+    compiler spilled there, a destination register could be saved before its load has landed, which
+    showed up as run-to-run differences when a variant of the kernel needed more registers than the
+    block size allows.  The committed kernel must therefore compile without any spill."""
+    import shutil
+    import subprocess
+    import tempfile
+    from paper_2502_17599_b200 import build
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    with tempfile.TemporaryDirectory() as tmp:
+        cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "--expt-relaxed-constexpr",
+               "-Xptxas", "-v", "-cubin", "-o", os.path.join(tmp, "meda.cubin")] + build.sources()
+        res = subprocess.run(cmd, capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+    lines = (res.stdout + res.stderr).splitlines()
+    hits = [i for i, line in enumerate(lines) if "Function properties" in line and "nearest_kernel" in line]
+    assert hits, "nearest_kernel not found in the ptxas report"
+    for i in hits:
+        assert "0 bytes spill stores, 0 bytes spill loads" in lines[i + 1], lines[i + 1]

@@ -38,6 +38,20 @@ def test_full_size_pass_sampled_against_the_oracle(name):
     cp.ctx.check()
     torch.cuda.synchronize()
 
+    # ---- a second run of the same pass gives the same bits everywhere (no float atomics, no races)
+    first = [t.clone() for t in (cp.entropy, cp.budgets, cp.scores)]
+    live = lambda: [torch.cat([x[l, :, : int(cp.budgets[l, 0])].reshape(-1).view(torch.uint8) for l in range(L)])
+                    for x in (cp.k_out, cp.v_out, cp.counts, cp.idx_c)]
+    first_live = live()
+    cp.run(qs, ks, vs)
+    cp.ctx.check()
+    torch.cuda.synchronize()
+    for a, b_ in zip(first, (cp.entropy, cp.budgets, cp.scores)):
+        assert torch.equal(a, b_)
+    for a, b_ in zip(first_live, live()):
+        assert torch.equal(a, b_)
+    del first, first_live
+
     # ---- budgets: bit-exact from the entropies the device produced; they sum to the global budget
     ent = P.np64(cp.entropy)
     budgets = cp.budgets.cpu().numpy()

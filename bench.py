@@ -204,6 +204,23 @@ def algorithmic_work(wl, budgets):
     return out
 
 
+# DRAM traffic of one launch of the arg-max kernel, dram__bytes_read.sum + dram__bytes_write.sum from the
+# ncu capture summarised in profiles/hot_kernels_long_video_128k_first2layers.md (134.3 MB read: the key
+# cache once, whatever the budget, plus the gathered keys; 4.6 MB written).  It is reported only while
+# the kernel's sources still hash to what was captured.
+NEAREST_TRAFFIC_BYTES = 138.9e6
+NEAREST_SOURCES = ("paper_2502_17599_b200/csrc/nearest_sm100.cuh", "paper_2502_17599_b200/csrc/sm100_primitives.cuh")
+NEAREST_SOURCES_SHA = "4443e42af73fb23c"
+
+
+def nearest_traffic():
+    import hashlib
+    h = hashlib.sha256()
+    for f in NEAREST_SOURCES:
+        h.update(open(os.path.join(ROOT, f), "rb").read())
+    return NEAREST_TRAFFIC_BYTES if h.hexdigest()[:16] == NEAREST_SOURCES_SHA else None
+
+
 def rank_workload(name, rank, layers=0):
     """The prompt rank `rank` compresses: the named workload with its own seed (independent prompts, so
     N ranks do N times the work: weak scaling, no data-path collective)."""
@@ -344,8 +361,10 @@ def run_ours(args):
         achieved = flops / (per_class["nearest"]["ms_per_step"] * 1e-3) / 1e12
         roof = {"kernel": "nearest (merge similarity + arg-max)", "bound": "tensor", "achieved": achieved,
                 "peak": pk["bf16_sustained"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"],
-                "traffic": None, "peak_source": pk["source"] + " (sustained cuBLAS bf16)",
-                "flops_per_step": flops}
+                "traffic": nearest_traffic(), "traffic_unit": "bytes per launch (ncu, 2-layer capture of the same config)",
+                "peak_source": pk["source"] + " (sustained cuBLAS bf16)", "flops_per_step": flops,
+                "flops_per_launch": flops / max(per_class["nearest"]["launches_per_step"], 1),
+                "us_per_launch": 1e3 * per_class["nearest"]["ms_per_step"] / max(per_class["nearest"]["launches_per_step"], 1)}
     else:
         key = {"stats": "stats_bytes", "sweep": "sweep_bytes", "reduce": "reduce_bytes"}.get(dominant)
         nbytes = sum(work[key]) if key else 0.0
@@ -359,6 +378,13 @@ def run_ours(args):
         if name in per_class:
             gbs = sum(work[key]) / (per_class[name]["ms_per_step"] * 1e-3) / 1e9
             extra[name] = {"GB/s": gbs, "frac_of_copy_peak": gbs / pk["hbm_gbs"]}
+    # the two phase-A sweeps evaluate one exp2 per logit on the special-function units: 16 per clock per SM
+    exps = float(L) * wl.n_q_heads * wl.window * wl.n_tokens
+    sfu_peak = 148 * 16 * (clocks["sm_max_mhz"] or 1965.0) * 1e6 if clocks else None
+    for name in ("stats", "sweep"):
+        if name in per_class and sfu_peak:
+            rate = exps / (per_class[name]["ms_per_step"] * 1e-3)
+            extra[name].update({"exp2/s": rate, "frac_of_sfu_peak": rate / sfu_peak})
     if "nearest" in per_class:
         tf = sum(work["nearest_flops"]) / (per_class["nearest"]["ms_per_step"] * 1e-3) / 1e12
         extra["nearest"] = {"TFLOP/s": tf, "frac_of_sustained_bf16": tf / pk["bf16_sustained"]}

@@ -36,6 +36,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long_video_128k")
     ap.add_argument("--layers", type=int, default=0, help="keep only the first N layers (profiling captures); 0 = all")
+    ap.add_argument("--streams", type=int, default=2, help="streams (and contexts) the layers alternate between")
     ap.add_argument("--eager", action="store_true", help="time eager launches instead of a CUDA-graph replay of the pass")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -272,7 +273,7 @@ def run_ours(args):
         q, k, v = W.make_layer(wl, l, "cuda")
         qs.append(q); ks.append(k); vs.append(v)
     input_bytes = sum(t.numel() * t.element_size() for ts in (qs, ks, vs) for t in ts)
-    cp = CompressionPass(wl)
+    cp = CompressionPass(wl, n_streams=args.streams)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -288,10 +289,10 @@ def run_ours(args):
     step = cp.replay if not args.eager else (lambda: cp.run(qs, ks, vs))
     for _ in range(args.warmup):
         step()
-    cp.ctx.check()
+    cp.check()
     budgets = cp.budgets.cpu().numpy()[:, 0]
 
-    launches0 = cp.ctx.launch_count()
+    launches0 = cp.launch_count()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -303,18 +304,18 @@ def run_ours(args):
     ev1.record(stream)
     barrier()
     ms_total = ev0.elapsed_time(ev1)
-    launches = kernels_per_pass * args.steps if not args.eager else cp.ctx.launch_count() - launches0
-    cp.ctx.check()
+    launches = kernels_per_pass * args.steps if not args.eager else cp.launch_count() - launches0
+    cp.check()
 
     cp.ctx.profile_enable(True)
     barrier()
     for _ in range(args.steps):
-        cp.run(qs, ks, vs)
+        cp.run(qs, ks, vs, single_stream=True)      # one stream: a launch's events bracket that launch alone
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     prof = cp.ctx.profile_read()
     cp.ctx.profile_enable(False)
-    cp.ctx.check()
+    cp.check()
     ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
     value = whole_job_throughput(wl, world, ms_step)
 
@@ -402,7 +403,8 @@ def run_ours(args):
         "config": {"workload": wl.name, "shape": wl.description, "global_budget": wl.global_budget,
                    "input_bytes": input_bytes, "l2": "inputs larger than L2 (no flush needed)" if input_bytes > 256e6 else "inputs fit L2",
                    "parallelism": f"independent prompts x{world}",
-                   "launch": "eager launches" if args.eager else f"one CUDA-graph replay per step ({kernels_per_pass} kernels)"},
+                   "launch": ("eager launches" if args.eager else f"one CUDA-graph replay per step ({kernels_per_pass} kernels)")
+                             + f", layers alternate between {len(cp.contexts)} streams"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roof, "kernels": per_class, "kernel_rooflines": extra, "cpu_baseline": cpu,
         "budgets_min_max": [int(budgets.min()), int(budgets.max())],

@@ -17,14 +17,21 @@ class CompressionPass:
     `row_capacity` bounds S_l per layer (n_tokens is always safe; a smaller value saves memory and
     makes a layer whose budget exceeds it report MEDA_ERR_WORKSPACE)."""
 
-    def __init__(self, wl: Workload, row_capacity: int | None = None, device="cuda", **ctx_overrides):
+    def __init__(self, wl: Workload, row_capacity: int | None = None, device="cuda", n_streams: int = 2,
+                 **ctx_overrides):
         self.wl = wl
         self.device = device
-        self.ctx = binding.Context.for_workload(wl, **ctx_overrides)
+        # Layers are independent inside each phase, so they alternate between `n_streams` streams, each
+        # with its own context (scratch memory): the short, latency-bound kernels of one layer
+        # (selection, sort passes, scans, reductions of partials) then run beside the long kernels of
+        # the next instead of leaving the GPU idle.
+        self.contexts = [binding.Context.for_workload(wl, **ctx_overrides) for _ in range(max(1, n_streams))]
+        self.ctx = self.contexts[0]
+        self.streams = [torch.cuda.Stream(device=device) for _ in self.contexts] if len(self.contexts) > 1 else []
         n, hkv, hq, w, d, L = wl.n_tokens, wl.n_kv_heads, wl.n_q_heads, wl.window, wl.head_dim, wl.n_layers
         self.cap = n if row_capacity is None else int(row_capacity)
         f32, i32 = torch.float32, torch.int32
-        self.row_stats = torch.empty((hq, w, 4), dtype=f32, device=device)
+        self.row_stats = [torch.empty((hq, w, 4), dtype=f32, device=device) for _ in self.contexts]
         self.scores = torch.empty((L, hkv, n), dtype=f32, device=device)
         self.entropy = torch.zeros(L, dtype=f32, device=device)
         self.budgets = torch.zeros((L, 3), dtype=i32, device=device)
@@ -34,19 +41,56 @@ class CompressionPass:
         self.idx_c = torch.empty((L, hkv, self.cap), dtype=i32, device=device)
 
     def close(self):
-        self.ctx.close()
+        for c in self.contexts:
+            c.close()
 
-    def run(self, q_layers, k_layers, v_layers, stream=None):
-        """Enqueues the whole pass on `stream` (default: torch's current stream).  Inputs are lists
-        of per-layer device tensors.  Results stay on the device in this object's buffers."""
+    def check(self):
+        """Synchronises and raises if any context recorded a device-side error."""
+        torch.cuda.synchronize()
+        for c in self.contexts:
+            c.check()
+
+    def launch_count(self) -> int:
+        return sum(c.launch_count() for c in self.contexts)
+
+    def _fork(self, main):
+        ev = torch.cuda.Event()
+        ev.record(main)
+        for s in self.streams:
+            s.wait_event(ev)
+
+    def _join(self, main):
+        for s in self.streams:
+            ev = torch.cuda.Event()
+            ev.record(s)
+            main.wait_event(ev)
+
+    def run(self, q_layers, k_layers, v_layers, stream=None, single_stream=False):
+        """Enqueues the whole pass.  Inputs are lists of per-layer device tensors; results stay on the
+        device in this object's buffers.  The work is ordered after what `stream` (default: torch's
+        current stream) holds and `stream` waits for all of it.  With `single_stream` everything goes to
+        `stream` through the first context (used when every launch is timed on its own)."""
         L = self.wl.n_layers
-        c = self.ctx
+        main = stream if stream is not None else torch.cuda.current_stream()
+        if single_stream or not self.streams:
+            lanes = [(self.contexts[0], main, self.row_stats[0])]
+        else:
+            lanes = list(zip(self.contexts, self.streams, self.row_stats))
+            self._fork(main)
         for l in range(L):
-            c.window_scores(l, q_layers[l], k_layers[l], self.row_stats, self.scores[l], self.entropy, stream)
-        c.allocate_budgets(self.entropy, self.budgets, stream)
+            c, s, rs = lanes[l % len(lanes)]
+            c.window_scores(l, q_layers[l], k_layers[l], rs, self.scores[l], self.entropy, s)
+        if len(lanes) > 1:
+            self._join(main)
+        self.ctx.allocate_budgets(self.entropy, self.budgets, main)      # Eq. 7 needs every layer's entropy
+        if len(lanes) > 1:
+            self._fork(main)
         for l in range(L):
+            c, s, _ = lanes[l % len(lanes)]
             c.compress_layer(l, k_layers[l], v_layers[l], self.scores[l], self.budgets, self.k_out[l], self.v_out[l],
-                             self.counts[l], self.idx_c[l], self.cap, stream)
+                             self.counts[l], self.idx_c[l], self.cap, s)
+        if len(lanes) > 1:
+            self._join(main)
 
     def capture(self, q_layers, k_layers, v_layers):
         """Records the whole pass (every launch of `run` on these buffers) into a CUDA graph, after one
@@ -55,12 +99,12 @@ class CompressionPass:
         Returns the number of kernels in the graph."""
         self.run(q_layers, k_layers, v_layers)
         torch.cuda.synchronize()
-        before = self.ctx.launch_count()
+        before = self.launch_count()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             self.run(q_layers, k_layers, v_layers)
         self.graph = graph
-        self.graph_kernels = self.ctx.launch_count() - before
+        self.graph_kernels = self.launch_count() - before
         return self.graph_kernels
 
     def replay(self):

@@ -35,8 +35,7 @@ def test_full_size_pass_sampled_against_the_oracle(name):
         qs.append(q); ks.append(k); vs.append(v)
     cp = CompressionPass(wl)
     cp.run(qs, ks, vs)
-    cp.ctx.check()
-    torch.cuda.synchronize()
+    cp.check()
 
     # ---- a second run of the same pass gives the same bits everywhere (no float atomics, no races)
     first = [t.clone() for t in (cp.entropy, cp.budgets, cp.scores)]
@@ -44,8 +43,7 @@ def test_full_size_pass_sampled_against_the_oracle(name):
                     for x in (cp.k_out, cp.v_out, cp.counts, cp.idx_c)]
     first_live = live()
     cp.run(qs, ks, vs)
-    cp.ctx.check()
-    torch.cuda.synchronize()
+    cp.check()
     for a, b_ in zip(first, (cp.entropy, cp.budgets, cp.scores)):
         assert torch.equal(a, b_)
     for a, b_ in zip(first_live, live()):

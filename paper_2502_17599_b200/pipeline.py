@@ -17,7 +17,7 @@ class CompressionPass:
     `row_capacity` bounds S_l per layer (n_tokens is always safe; a smaller value saves memory and
     makes a layer whose budget exceeds it report MEDA_ERR_WORKSPACE)."""
 
-    def __init__(self, wl: Workload, row_capacity: int | None = None, device="cuda", n_streams: int = 2,
+    def __init__(self, wl: Workload, row_capacity: int | None = None, device="cuda", n_streams: int = 4,
                  **ctx_overrides):
         self.wl = wl
         self.device = device

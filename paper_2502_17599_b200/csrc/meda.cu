@@ -63,6 +63,14 @@ void free_workspace(Workspace& ws) {
   ws = Workspace();
 }
 
+// grid.x of a kernel that walks up to `slots` conserved slots with a stride, `per_block` slots per block
+// and step, replicated `copies` times in grid.y / grid.z: about sixteen blocks per SM in total.  The slot
+// count is only known on the device, so the grid is sized for the worst case and must stay small.
+int slot_blocks(const meda_ctx* ctx, int slots, int per_block, int copies) {
+  const int needed = (slots + per_block - 1) / per_block;
+  return std::max(1, std::min(needed, (ctx->sm_count * 16 + copies - 1) / copies));
+}
+
 int generic_tiles(int n) { return (n + kGenericKeyTile - 1) / kGenericKeyTile; }
 
 // Raises a kernel's dynamic shared memory limit to the most the SM offers next to the kernel's
@@ -289,7 +297,7 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
   const int max_slots = std::min(cap, n);
   {
     LaunchScope scope(ctx, MEDA_K_PREP, st);
-    gather_conserved_bf16_kernel<<<dim3(std::min((max_slots + 7) / 8, ctx->sm_count * 8), c.n_kv_heads), 256, 0, st>>>(
+    gather_conserved_bf16_kernel<<<dim3(slot_blocks(ctx, max_slots, 8, c.n_kv_heads), c.n_kv_heads), 256, 0, st>>>(
         static_cast<const __nv_bfloat16*>(k), idx_conserved, budget_row, ctx->ws.kc, ctx->ws.inv_norm, n, cap,
         ctx->kc_rows, ctx->inv_stride);
   }
@@ -319,7 +327,7 @@ void launch_seg_kernels(meda_ctx* ctx, const void* k, const void* v, const int32
         ctx->ws.carry_cnt, n, cap, ctx->seg_chunks);
   }
   LaunchScope scope(ctx, MEDA_K_REDUCE, st);
-  seg_finalize_kernel<T, D><<<dim3(std::min((max_slots + 7) / 8, ctx->sm_count * 8), c.n_kv_heads, 2), 256, 0, st>>>(
+  seg_finalize_kernel<T, D><<<dim3(slot_blocks(ctx, max_slots, 8, 2 * c.n_kv_heads), c.n_kv_heads, 2), 256, 0, st>>>(
       static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, budget_row, ctx->ws.seg_start,
       ctx->ws.seg_end, ctx->ws.carry, ctx->ws.carry_cnt, static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n,
       cap, ctx->seg_chunks, evict);
@@ -338,7 +346,7 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
   if (!evict) {
     {
       LaunchScope scope(ctx, MEDA_K_GROUP, st);
-      clear_segments_kernel<<<dim3(std::min((max_slots + 255) / 256, ctx->sm_count), c.n_kv_heads), 256, 0, st>>>(ctx->ws.seg_start,
+      clear_segments_kernel<<<dim3(slot_blocks(ctx, max_slots, 256, c.n_kv_heads), c.n_kv_heads), 256, 0, st>>>(ctx->ws.seg_start,
                                                                                        ctx->ws.seg_end, budget_row, n, cap);
     }
     const dim3 grid(ctx->sort_chunks, c.n_kv_heads);

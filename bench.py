@@ -211,7 +211,7 @@ def algorithmic_work(wl, budgets):
 # the kernel's sources still hash to what was captured.
 NEAREST_TRAFFIC_BYTES = 138.9e6
 NEAREST_SOURCES = ("paper_2502_17599_b200/csrc/nearest_sm100.cuh", "paper_2502_17599_b200/csrc/sm100_primitives.cuh")
-NEAREST_SOURCES_SHA = "4443e42af73fb23c"
+NEAREST_SOURCES_SHA = "69a1b0a6fffe1d3c"
 
 
 def nearest_traffic():

@@ -94,50 +94,11 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t columns) {
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// Same contraction with the A operand in tensor memory: lane r of the 128 lanes holds row r, column
-// c of the operand holds the bf16 pair (k = 2c, 2c + 1); one instruction consumes 8 columns (K = 16).
-__device__ __forceinline__ void umma_bf16_a_tmem(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
-                                                 uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 // Makes `bar` complete one arrival when every UMMA issued so far by this thread has finished.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base lane + t).
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
 // 32 lanes x 32 consecutive 32-bit columns, registers -> tensor memory: thread t of the warp writes
 // lane (base lane + t).  tmem_st_wait completes every store this thread has issued.
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -199,24 +160,19 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 
 // Shared-memory operand descriptor of a K-major bf16 tile stored as rows of 64 elements (128 bytes)
 // with the 128-byte swizzle a TMA load with CU_TENSOR_MAP_SWIZZLE_128B produces; the tile base must
-// be 1024-byte aligned.  Eight rows form one 1024-byte swizzle atom (stride-byte-offset field);
-// `byte_offset` selects the 16-element K slice inside the 128-byte row (0, 32, 64, 96).
-__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t tile_smem_addr, uint32_t byte_offset) {
-  const uint32_t addr = tile_smem_addr + byte_offset;
-  uint64_t lo = (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)1u << 16);          // start address, LBO = 1 (unused)
-  uint64_t hi = (uint64_t)(1024u >> 4) | ((uint64_t)1u << 14) | ((uint64_t)2u << 29);  // SBO, version 1, SWIZZLE_128B
-  return lo | (hi << 32);
-}
-
-// The same descriptor in two 32-bit halves, for issue loops: the high half is a constant and moving
-// the start address by `bytes` (a multiple of 16, inside the same tile) adds bytes / 16 to the low
-// half, so one integer add per operand replaces rebuilding the descriptor for every instruction.
-// The single thread that issues the UMMAs must spend fewer cycles per instruction than the tensor
-// pipe takes to run it (N / 2 cycles), or it becomes the bottleneck of the whole kernel.
+// be 1024-byte aligned.  Eight rows form one 1024-byte swizzle atom (stride-byte-offset field).  The
+// 64-bit descriptor is kept as two 32-bit halves: the high half (stride, version, swizzle mode) is
+// a constant, the low half holds (start address / 16) in its low 14 bits plus a fixed leading-offset
+// field, so moving the start address by `bytes` (a multiple of 16, inside the same tile) adds
+// bytes / 16 to the low half: one integer add per operand per instruction.  The K slice of an
+// instruction (16 elements) is 32 bytes inside the 128-byte row.
+// The thread that issues the UMMAs must spend fewer cycles per instruction than the tensor pipe
+// takes to run it, or it becomes the bottleneck of the whole kernel.
 constexpr uint32_t kUmmaDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t umma_desc_lo_sw128(uint32_t tile_smem_addr) {
   return ((tile_smem_addr >> 4) & 0x3FFFu) | (1u << 16);
 }
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, issued by one thread.
 __device__ __forceinline__ void umma_bf16_lohi(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
                                                uint32_t accumulate) {
   asm volatile(
@@ -228,6 +184,8 @@ __device__ __forceinline__ void umma_bf16_lohi(uint32_t tmem_d, uint32_t a_lo, u
       ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(kUmmaDescHiSw128), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same contraction with the A operand in tensor memory: lane r of the 128 lanes holds row r, column
+// c of the operand holds the bf16 pair (k = 2c, 2c + 1); one instruction consumes 8 columns (K = 16).
 __device__ __forceinline__ void umma_bf16_a_tmem_lohi(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t idesc,
                                                       uint32_t accumulate) {
   asm volatile(

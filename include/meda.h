@@ -111,12 +111,18 @@ meda_status meda_poll_status(meda_ctx* ctx, void* stream);
 meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
                                float* row_stats, float* scores, float* entropy, void* stream);
 
-/* Cross-modal attention entropy of one layer from existing row_stats (Eq. 4-6): one sweep over
- * the key cache, writes entropy[layer].  For callers that already hold the normalisers.
- * q_vis / q_vis_pos / n_vis_rows describe an optional window of VISUAL query rows
- * ([n_q_heads][n_vis_rows][head_dim] and their absolute positions) for the E_VT term of Eq. 5;
- * pass NULL, NULL, 0 for the text-window-only definition E_CM = -E_TV.  A non-NULL q_vis
- * returns MEDA_ERR_UNSUPPORTED in this build. */
+/* Cross-modal attention entropy of one layer (Eq. 4-6): E_CM = -(E_TV + E_VT), written to entropy[layer].
+ *  - The E_TV term uses the text window q_win and its row_stats (from meda_window_scores): one sweep over
+ *    the key cache, the same arithmetic as meda_window_scores' own entropy.  For callers that already hold
+ *    the normalisers.
+ *  - The E_VT term of Eq. 5 needs VISUAL query rows, which a text window does not contain: q_vis (device,
+ *    `dtype`, [n_q_heads][n_vis_rows][head_dim]) and q_vis_pos (device int32 [n_vis_rows], the rows'
+ *    absolute token positions, each seeing the keys at or before it).  Its softmax is taken over the TEXT keys
+ *    a row sees; rows that see no text key are left out of the mean, as are they from its divisor.  With these
+ *    two sweeps over the text keys -E_VT is added to entropy[layer].  n_vis_rows <= 128.  Pass NULL, NULL, 0
+ *    for the text-window-only definition E_CM = -E_TV.
+ *  - q_win (and row_stats) may be NULL when q_vis is given: then only -E_VT is added to what entropy[layer]
+ *    already holds (for example the value meda_window_scores wrote). */
 meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
                                const float* row_stats, const void* q_vis, const int32_t* q_vis_pos,
                                int32_t n_vis_rows, float* entropy, void* stream);

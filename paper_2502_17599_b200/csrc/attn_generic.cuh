@@ -43,7 +43,7 @@ __device__ __forceinline__ void stage_k(float* ks, const T* k_g, int j0, int n, 
 // s[i][jl] = scale * q_i . k_jl for the staged tile; -inf where the key is past the end of the
 // sequence or hidden from row i by the causal mask.
 __device__ __forceinline__ void tile_logits(float* s, const float* qs, const float* ks, int w, int d,
-                                            int j0, int n, float scale) {
+                                            int j0, int n, float scale, const int32_t* __restrict__ q_pos = nullptr) {
   const int jl = threadIdx.x % kGenericKeyTile;
   const int ig = threadIdx.x / kGenericKeyTile;           // 0..3
   constexpr int kRowStep = kAttnThreads / kGenericKeyTile;
@@ -54,7 +54,7 @@ __device__ __forceinline__ void tile_logits(float* s, const float* qs, const flo
     float acc = 0.f;
 #pragma unroll 8
     for (int t = 0; t < d; ++t) acc = fmaf(qr[t], kr[t], acc);
-    bool visible = (j < n) && (j <= n - w + i);
+    bool visible = (j < n) && (j <= (q_pos ? q_pos[i] : n - w + i));      // default rows: the last w tokens
     s[i * kGenericKeyTile + jl] = visible ? acc * scale : -INFINITY;
   }
 }
@@ -66,7 +66,8 @@ __device__ __forceinline__ void tile_logits(float* s, const float* qs, const flo
 template <typename T>
 __global__ void __launch_bounds__(kAttnThreads)
 stats_partial_kernel(const T* __restrict__ q_win, const T* __restrict__ k, const uint8_t* __restrict__ modality,
-                     float* __restrict__ partial, int hq, int group, int n, int w, int d, float scale) {
+                     float* __restrict__ partial, int hq, int group, int n, int w, int d, float scale,
+                     const int32_t* __restrict__ q_pos = nullptr, int subset = MEDA_VISUAL, int subset_only = 0) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const AttnGenericSmem L = attn_generic_smem(w, d, false);
   float* qs = reinterpret_cast<float*>(smem_raw + L.q_off);
@@ -89,14 +90,20 @@ stats_partial_kernel(const T* __restrict__ q_win, const T* __restrict__ k, const
 
   for (int tile = blockIdx.x; tile < n_tiles; tile += chunks) {
     const int j0 = tile * kGenericKeyTile;
+    if (subset_only) {
+      // only the restricted normaliser is wanted: a tile without a key of the subset contributes nothing
+      const int jj = j0 + (int)threadIdx.x;
+      const int mine = (threadIdx.x < kGenericKeyTile && jj < n && modality[jj] == subset) ? 1 : 0;
+      if (!__syncthreads_or(mine)) continue;
+    }
     stage_k<T>(ks, k_g, j0, n, d);
     __syncthreads();
-    tile_logits(s, qs, ks, w, d, j0, n, scale);
+    tile_logits(s, qs, ks, w, d, j0, n, scale, q_pos);
     __syncthreads();
     for (int i = warp; i < w; i += kAttnThreads / 32) {
       float a0 = s[i * kGenericKeyTile + lane], a1 = s[i * kGenericKeyTile + lane + 32];
-      bool v0 = (j0 + lane < n) && modality[min(j0 + lane, n - 1)] == MEDA_VISUAL;
-      bool v1 = (j0 + lane + 32 < n) && modality[min(j0 + lane + 32, n - 1)] == MEDA_VISUAL;
+      bool v0 = (j0 + lane < n) && modality[min(j0 + lane, n - 1)] == subset;
+      bool v1 = (j0 + lane + 32 < n) && modality[min(j0 + lane + 32, n - 1)] == subset;
       float b0 = v0 ? a0 : -INFINITY, b1 = v1 ? a1 : -INFINITY;
       float m_all = warp_max(fmaxf(a0, a1));
       float m_vis = warp_max(fmaxf(b0, b1));
@@ -158,7 +165,8 @@ __global__ void __launch_bounds__(kAttnThreads)
 scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, const uint8_t* __restrict__ modality,
                       const float* __restrict__ row_stats, float* __restrict__ scores,
                       float* __restrict__ ent_partial, int hq, int group, int n, int w, int d, float scale,
-                      int entropy_mode, int want_scores, int want_entropy) {
+                      int entropy_mode, int want_scores, int want_entropy,
+                      const int32_t* __restrict__ q_pos = nullptr, int subset = MEDA_VISUAL) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const AttnGenericSmem L = attn_generic_smem(w, d, true);
   float* qs = reinterpret_cast<float*>(smem_raw + L.q_off);
@@ -174,8 +182,13 @@ scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, cons
   constexpr int kRowStep = kAttnThreads / kGenericKeyTile;
   const int j = j0 + jl;
   const bool in_range = j < n;
-  const bool visual = in_range && modality[in_range ? j : 0] == MEDA_VISUAL;
+  const bool visual = in_range && modality[in_range ? j : 0] == subset;      // "in the subset the entropy is taken over"
   const float inv_hq = 1.f / (float)hq;
+  if (!want_scores && !__syncthreads_or(visual ? 1 : 0)) {
+    // entropy only, and no key of this tile is in the subset: nothing to add
+    if (threadIdx.x == 0) ent_partial[blockIdx.x] = 0.f;
+    return;
+  }
 
   for (int e = threadIdx.x; e < w * kGenericKeyTile; e += blockDim.x) abar[e] = 0.f;
   float plogp = 0.f;     // entropy_mode 1 accumulator
@@ -187,14 +200,14 @@ scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, cons
     stage_q<T>(qs, q_win + (size_t)h * w * d, w, d);
     if (h % group == 0) stage_k<T>(ks, k + (size_t)g * n * d, j0, n, d);
     __syncthreads();
-    tile_logits(s, qs, ks, w, d, j0, n, scale);
+    tile_logits(s, qs, ks, w, d, j0, n, scale, q_pos);
     // each thread revisits only the logits it wrote itself: no barrier needed here
     float part = 0.f;
     for (int i = ig; i < w; i += kRowStep) {
       const float* rsp = row_stats + ((size_t)h * w + i) * 4;
       float sv = s[i * kGenericKeyTile + jl];
       if (sv > -INFINITY) {
-        part += expf(sv - rsp[0]) / rsp[1];
+        if (want_scores) part += expf(sv - rsp[0]) / rsp[1];
         if (visual && want_entropy) {
           float pv = expf(sv - rsp[2]) / rsp[3];
           if (entropy_mode == 0) abar[i * kGenericKeyTile + jl] += pv * inv_hq;
@@ -237,7 +250,8 @@ scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, cons
 // entropy[layer] = -(1 / rows) * sum of the partials in index order (fixed-shape reduction, so
 // repeated runs give identical bits).  rows = window rows that see at least one visual key.
 __global__ void entropy_finalize_kernel(const float* __restrict__ ent_partial, int n_partials,
-                                        const float* __restrict__ row_stats, int w, float* __restrict__ entropy_out) {
+                                        const float* __restrict__ row_stats, int w, float* __restrict__ entropy_out,
+                                        int accumulate = 0) {
   __shared__ double red[256];
   double acc = 0.0;
   for (int e = threadIdx.x; e < n_partials; e += blockDim.x) acc += (double)ent_partial[e];
@@ -250,7 +264,8 @@ __global__ void entropy_finalize_kernel(const float* __restrict__ ent_partial, i
   if (threadIdx.x == 0) {
     int rows = 0;
     for (int i = 0; i < w; ++i) rows += (row_stats[i * 4 + 3] > 0.f) ? 1 : 0;   // head 0
-    *entropy_out = rows > 0 ? (float)(-red[0] / (double)rows) : 0.f;
+    const float term = rows > 0 ? (float)(-red[0] / (double)rows) : 0.f;
+    *entropy_out = accumulate ? *entropy_out + term : term;      // E_CM = (-E_TV) + (-E_VT), Eq. 6
   }
 }
 

@@ -47,6 +47,7 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.modality);
   cudaFree(ws.status);
   cudaFree(ws.stats_partial);
+  cudaFree(ws.row_stats_vis);
   cudaFree(ws.ent_partial);
   cudaFree(ws.inv_norm);
   cudaFree(ws.target);
@@ -281,6 +282,43 @@ meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, c
     LaunchScope scope(ctx, MEDA_K_ENTROPY_FINAL, st);
     entropy_finalize_kernel<<<1, 256, 0, st>>>(ctx->ws.ent_partial, ((c.n_tokens + 255) / 256) * kUsEpilogueWarps,
                                                row_stats, c.window, entropy + layer);
+  }
+  return launch_status();
+}
+
+// The E_VT term of Eq. 5-6 on the CUDA-core kernels, any dtype: visual query rows at given positions
+// against the TEXT keys they see.  Adds -E_VT to entropy[layer].
+template <typename T>
+meda_status launch_evt(meda_ctx* ctx, int32_t layer, const void* q_vis, const int32_t* q_vis_pos, int32_t rows,
+                       const void* k, float* entropy, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const float scale = 1.0f / sqrtf((float)c.head_dim);
+  const int tiles = generic_tiles(c.n_tokens);
+  const int chunks = std::min(kStatsChunks, tiles);
+  const int stats_smem = attn_generic_smem(rows, c.head_dim, false).total;
+  const int sweep_smem = attn_generic_smem(rows, c.head_dim, true).total;
+  if (sweep_smem > kMaxDynSmem - 4096) return MEDA_ERR_SHAPE;
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS, st);
+    stats_partial_kernel<T><<<dim3(chunks, c.n_q_heads), kAttnThreads, stats_smem, st>>>(
+        static_cast<const T*>(q_vis), static_cast<const T*>(k), ctx->ws.modality, ctx->ws.stats_partial, c.n_q_heads,
+        ctx->group, c.n_tokens, rows, c.head_dim, scale, q_vis_pos, MEDA_TEXT, 1);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
+    stats_combine_kernel<<<(c.n_q_heads * rows + 7) / 8, 256, 0, st>>>(ctx->ws.stats_partial, ctx->ws.row_stats_vis, chunks,
+                                                                       c.n_q_heads * rows);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_SWEEP, st);
+    scores_entropy_kernel<T><<<tiles, kAttnThreads, sweep_smem, st>>>(
+        static_cast<const T*>(q_vis), static_cast<const T*>(k), ctx->ws.modality, ctx->ws.row_stats_vis, nullptr,
+        ctx->ws.ent_partial, c.n_q_heads, ctx->group, c.n_tokens, rows, c.head_dim, scale, c.entropy_mode, 0, 1,
+        q_vis_pos, MEDA_TEXT);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_ENTROPY_FINAL, st);
+    entropy_finalize_kernel<<<1, 256, 0, st>>>(ctx->ws.ent_partial, tiles, ctx->ws.row_stats_vis, rows, entropy + layer, 1);
   }
   return launch_status();
 }
@@ -564,8 +602,12 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   if (st == MEDA_OK) st = carve(&ws.modality, mod_bytes, &ws.bytes);
   if (st == MEDA_OK && cudaMemset(ws.modality, 2, (size_t)mod_bytes) != cudaSuccess) st = MEDA_ERR_CUDA;
   if (st == MEDA_OK) st = carve(&ws.status, 1, &ws.bytes);
+  // the partial normalisers also serve the visual query window of meda_layer_entropy (up to kMaxWindow rows)
   if (st == MEDA_OK)
-    st = carve(&ws.stats_partial, (int64_t)std::max(kStatsChunks, ctx->stats_chunks * StatsPolicy::kEpilogueGroups) * c.n_q_heads * c.window * 4, &ws.bytes);
+    st = carve(&ws.stats_partial,
+               std::max((int64_t)std::max(kStatsChunks, ctx->stats_chunks * StatsPolicy::kEpilogueGroups) * c.n_q_heads * c.window * 4,
+                        (int64_t)kStatsChunks * c.n_q_heads * kMaxWindow * 4), &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.row_stats_vis, (int64_t)c.n_q_heads * kMaxWindow * 4, &ws.bytes);
   if (ctx->fast_attn) {
     if (st == MEDA_OK) st = carve(&ws.coef_vis, (int64_t)c.n_q_heads * c.window, &ws.bytes);
     if (st == MEDA_OK) st = carve(&ws.coef_text, (int64_t)c.n_q_heads * c.window, &ws.bytes);
@@ -716,12 +758,23 @@ meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, 
 meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
                                const void* q_vis, const int32_t* q_vis_pos, int32_t n_vis_rows, float* entropy,
                                void* stream) {
-  if (!layer_ok(ctx, layer) || !q_win || !k || !row_stats || !entropy) return MEDA_ERR_INVALID_ARG;
-  if (q_vis || q_vis_pos || n_vis_rows != 0) return MEDA_ERR_UNSUPPORTED;
+  if (!layer_ok(ctx, layer) || !k || !entropy) return MEDA_ERR_INVALID_ARG;
+  const bool with_vis = q_vis || q_vis_pos || n_vis_rows != 0;
+  if (with_vis && (!q_vis || !q_vis_pos || n_vis_rows < 1)) return MEDA_ERR_INVALID_ARG;
+  if (with_vis && n_vis_rows > kMaxWindow) return MEDA_ERR_SHAPE;
+  if (!q_win && !with_vis) return MEDA_ERR_INVALID_ARG;          // nothing to compute
+  if (q_win && !row_stats) return MEDA_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
-  if (ctx->fast_attn) return launch_sweep_fast(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
-  if (ctx->cfg.dtype == MEDA_F32) return launch_sweep<float>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
-  return launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
+  meda_status r = MEDA_OK;
+  if (q_win) {
+    if (ctx->fast_attn) r = launch_sweep_fast(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
+    else if (ctx->cfg.dtype == MEDA_F32) r = launch_sweep<float>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
+    else r = launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
+  }
+  if (r == MEDA_OK && with_vis)
+    r = ctx->cfg.dtype == MEDA_F32 ? launch_evt<float>(ctx, layer, q_vis, q_vis_pos, n_vis_rows, k, entropy, st)
+                                   : launch_evt<__nv_bfloat16>(ctx, layer, q_vis, q_vis_pos, n_vis_rows, k, entropy, st);
+  return r;
 }
 
 meda_status meda_allocate_budgets(meda_ctx* ctx, const float* entropy, int32_t* budgets, void* stream) {

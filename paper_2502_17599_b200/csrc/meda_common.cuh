@@ -22,6 +22,7 @@ struct Workspace {
   float2* coef_text = nullptr;        // [Hq * w]
   int* status = nullptr;              // device status word (first error wins)
   float* stats_partial = nullptr;     // [chunks][Hq][w][4]
+  float* row_stats_vis = nullptr;     // [Hq][<= kMaxWindow][4] normalisers of the visual query window (E_VT)
   float* ent_partial = nullptr;       // [ent_slots]
   float* inv_norm = nullptr;          // [Hkv][inv_stride]  1 / max(|k_c|, eps) per conserved slot
   __nv_bfloat16* kc = nullptr;        // [Hkv][kc_rows][128] gathered conserved keys (bf16, head_dim 128 only)

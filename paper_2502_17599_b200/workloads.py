@@ -233,3 +233,19 @@ def make_layer(wl: Workload, layer: int, device="cpu"):
     tau = layer_temperature(wl, layer)
     q = (tau * normal(stream_key(wl.seed, layer, 2), 0, hq * w * d, device)).view(hq, w, d).to(wl.torch_dtype)
     return q, k, v
+
+
+def make_visual_queries(wl: Workload, layer: int, n_rows: int, device="cpu"):
+    """(q_vis [Hq, n_rows, d] in the workload's dtype, positions int32 [n_rows]): query rows of `n_rows`
+    visual tokens spread evenly over the prompt's visual tokens, for the vision-to-text term of the
+    cross-modal entropy.  Same distribution as the text window's queries (one temperature per layer)."""
+    vis = torch.nonzero(wl.modality("cpu") == VISUAL).flatten()
+    if vis.numel() == 0:
+        raise ValueError("the workload has no visual token")
+    pick = torch.linspace(0, vis.numel() - 1, n_rows).round().to(torch.int64)
+    pos = vis[pick].to(torch.int32).to(device)
+    hq, d = wl.n_q_heads, wl.head_dim
+    tau = layer_temperature(wl, layer)
+    q = (tau * normal(stream_key(wl.seed, layer, 3), 0, hq * n_rows * d, device)).view(hq, n_rows, d).to(wl.torch_dtype)
+    return q, pos
+

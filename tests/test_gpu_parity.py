@@ -312,3 +312,35 @@ def test_select_beyond_cluster_capacity_uses_the_single_block_kernel():
         less = idx_l[0, : n - M - N].cpu().numpy()
         assert (np.diff(less) > 0).all() and less.size + M + N == n
     ctx.close()
+
+
+@pytest.mark.parametrize("wl", [
+    W.small_variant(),                                                          # CUDA-core kernels for both terms
+    W.small_variant("evt_tc_w32", window=32, seed=4),                           # E_TV on the tensor cores, E_VT on CUDA cores
+    W.small_variant("evt_f32", dtype="f32", n_q_heads=4, n_kv_heads=2, head_dim=64, seed=3),
+    # the prompt opens with an image: its first visual rows see no text key and drop out of the mean
+    W.small_variant("evt_visual_first", spans=((0, 200, 1), (200, 260, 0), (260, 600, 1), (600, 661, 0)), frame_tokens=0, seed=8),
+], ids=lambda w: w.name)
+@pytest.mark.parametrize("entropy_mode", [0, 1])
+def test_cross_modal_entropy_with_the_vision_to_text_term(wl, entropy_mode):
+    """E_CM = -(E_TV + E_VT) of Eq. 5-6 with a window of visual query rows, in one call and in two."""
+    ctx = make_ctx(wl, entropy_mode=entropy_mode)
+    buf = P.GpuBuffers(wl)
+    mod = wl.modality().numpy()
+    n_rows = 19
+    for l in range(2):
+        (q, k, v), (qh, kh, vh) = P.layer_inputs(wl, l, "cuda")
+        qv, pos = W.make_visual_queries(wl, l, n_rows, "cuda")
+        want = O.cross_modal_entropy(qh, kh, mod, q_vis=P.np64(qv), q_vis_pos=pos.cpu().numpy().astype(np.int64),
+                                     entropy_mode=entropy_mode)
+        want_tv = O.cross_modal_entropy(qh, kh, mod, entropy_mode=entropy_mode)
+        assert abs(want - want_tv) > 1e-3                     # the extra term is really there
+        ctx.window_scores(l, q, k, buf.row_stats, buf.scores, buf.entropy)        # writes -E_TV
+        both = torch.zeros_like(buf.entropy)
+        ctx.layer_entropy(l, q, k, buf.row_stats, both, q_vis=qv, q_vis_pos=pos, n_vis_rows=n_rows)
+        ctx.layer_entropy(l, None, k, None, buf.entropy, q_vis=qv, q_vis_pos=pos, n_vis_rows=n_rows)   # adds -E_VT
+        ctx.check()
+        P.assert_entropy_close(float(both[l]), want)
+        assert float(buf.entropy[l]) == float(both[l])
+    ctx.close()
+

@@ -177,23 +177,22 @@ struct StatsPolicy {
 };
 
 // ---------------------------------------------------------------------------------------------
-// Per-column constants of sweep 2, from the normalisers.
-//   vis[c]  = (m_vis * log2e, exp(m_vis - m_all) / z_all, 1 / (z_vis * Hq), -ln z_vis)   for visual keys
-//   text[c] = (m_all * log2e, 1 / z_all)                                                  for text keys
-// so that one e = exp2(t - ref) gives the full-softmax probability e * [1] and, for a visual key,
-// the head-averaged visual-softmax probability e * [2].
+// Per-column constants of sweep 2, from the normalisers (column = query head * w + window row).
+//   vis[c]  = (m_vis * log2e + log2(z_vis * Hq),  Hq * z_vis * exp(m_vis - m_all) / z_all)   for visual keys
+//   text[c] = (m_all * log2e,                     1 / z_all)                                 for text keys
+// For a visual key one e = exp2(t - vis.x) is already the head-averaged visual-softmax probability
+// p_vis / Hq, and e * vis.y is the full-softmax probability; for a text key exp2(t - text.x) * text.y
+// is the full-softmax probability.  A row that sees no visual key gets (+huge, 0): e = 0.
 // ---------------------------------------------------------------------------------------------
-__global__ void sweep_coef_kernel(const float* __restrict__ row_stats, float4* __restrict__ vis,
-                                  float2* __restrict__ text, int rows, float inv_hq) {
+__global__ void sweep_coef_kernel(const float* __restrict__ row_stats, float2* __restrict__ vis,
+                                  float2* __restrict__ text, int rows, float hq) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= rows) return;
   const float4 s = reinterpret_cast<const float4*>(row_stats)[c];
-  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  float2 a = make_float2(1e30f, 0.f);
   if (s.w > 0.f) {
-    a.x = s.z * kLog2e;
-    a.y = expf(s.z - s.x) / s.y;
-    a.z = inv_hq / s.w;
-    a.w = -logf(s.w);
+    a.x = fmaf(s.z, kLog2e, log2f(s.w * hq));
+    a.y = hq * s.w * expf(s.z - s.x) / s.y;
   }
   vis[c] = a;
   text[c] = make_float2(s.x * kLog2e, 1.f / s.y);
@@ -210,20 +209,21 @@ template <int W, int MODE>
 struct SweepPolicy {
   struct Params {
     const uint8_t* modality;     // padded as above
-    const float4* vis;           // [Hq * w]
+    const float2* vis;           // [Hq * w]
     const float2* text;          // [Hq * w]
     float* scores;               // [Hkv][n] or null
     float* ent_partial;          // [blocks * 8] or null
     int n, hkv, cols;            // cols = group * W columns per KV head (multiple of 32, <= kSweepMaxCols)
     int n_blocks;                // ceil(n / 256)
     float sc2;
+    float ln_hq;                 // ln(n_q_heads): ln p = ln(p / Hq) + ln Hq in the mean of per-head entropies
   };
   static constexpr int kABuffers = 2;
   static constexpr int kBStages = 2;
   static constexpr int kEpilogueGroups = 1;
   static constexpr uint32_t kExtraBytes = 0;
-  static constexpr uint32_t kTextOff = kSweepMaxCols * 16;
-  static constexpr uint32_t kItemExtraBytes = kSweepMaxCols * (16 + 8);
+  static constexpr uint32_t kTextOff = kSweepMaxCols * 8;
+  static constexpr uint32_t kItemExtraBytes = kSweepMaxCols * (8 + 8);
 
   __device__ static bool active(const Params&) { return true; }
   // Each block takes whole 256-key blocks and walks all KV heads of a block back to back, so that
@@ -243,19 +243,21 @@ struct SweepPolicy {
     o.u1 = blk;
     return true;
   }
-  __device__ static uint32_t item_extra_bytes(const Params& p, const StreamItem&) { return (uint32_t)p.cols * 24u; }
+  __device__ static uint32_t item_extra_bytes(const Params& p, const StreamItem&) { return (uint32_t)p.cols * 16u; }
   __device__ static void item_extra_issue(const Params& p, const StreamItem& it, unsigned char* dst, uint64_t* bar) {
-    sm100::bulk_load(dst, p.vis + it.b_row, (uint32_t)p.cols * 16u, bar);
+    sm100::bulk_load(dst, p.vis + it.b_row, (uint32_t)p.cols * 8u, bar);
     sm100::bulk_load(dst + kTextOff, p.text + it.b_row, (uint32_t)p.cols * 8u, bar);
   }
 
   struct Epilogue {
     int lane, ewarp, row_in_block;
-    const float4* cvis;          // this item's constants, shared memory
-    const float2* ctext;
+    const float4* cvis;          // this item's constants in shared memory, two columns per 16 bytes
+    const float4* ctext;
     float abar[W];               // head-averaged visual-softmax attention of this key, per window row
     float plogp;                 // MODE 1 accumulator
     float score;
+    int md, first_row;           // this thread's key: modality, first window row that sees it
+    bool valid, masked;
     __device__ void init(const Params&, unsigned char*, int ewarp_, int lane_) {
       lane = lane_;
       ewarp = ewarp_;
@@ -264,81 +266,89 @@ struct SweepPolicy {
       for (int x = 0; x < W; ++x) abar[x] = 0.f;
       plogp = 0.f;
     }
-    __device__ void item_begin(const Params&, const StreamItem&, const unsigned char* item_extra) {
+    __device__ void item_begin(const Params& p, const StreamItem& it, const unsigned char* item_extra) {
       score = 0.f;
       cvis = reinterpret_cast<const float4*>(item_extra);
-      ctext = reinterpret_cast<const float2*>(item_extra + kTextOff);
+      ctext = reinterpret_cast<const float4*>(item_extra + kTextOff);
+      // what the tiles need to know about this thread's key, fetched once per item, off the tile path
+      const int j = it.a_row + row_in_block;
+      valid = j < p.n;
+      md = p.modality[j];                                  // the padded map covers j up to the block end
+      first_row = j - (p.n - W);                           // causal: window rows i >= first_row see key j
+      masked = __any_sync(0xffffffffu, valid && first_row > 0);
     }
 
     // A visual key against 32 query columns (one head's window rows OFF .. OFF + 31), all of which see it.
     template <int OFF>
     __device__ __forceinline__ void chunk_visual(const Params& p, const uint32_t (&r)[32], const float4* c4) {
 #pragma unroll
-      for (int x = 0; x < 32; ++x) {
-        const float4 c = c4[x];
-        const float t = fmaf(__uint_as_float(r[x]), p.sc2, -c.x);
-        const float e = fast_exp2(t);
-        score = fmaf(e, c.y, score);
-        if (MODE == 0) abar[OFF + x] = fmaf(e, c.z, abar[OFF + x]);
-        else plogp = fmaf(e * c.z, fmaf(t, kLn2, c.w), plogp);
+      for (int x = 0; x < 32; x += 2) {
+        const float4 c = c4[x / 2];                        // (ref, ratio) of columns x and x + 1
+        const float t0 = fmaf(__uint_as_float(r[x]), p.sc2, -c.x);
+        const float t1 = fmaf(__uint_as_float(r[x + 1]), p.sc2, -c.z);
+        const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
+        score = fmaf(e0, c.y, score);
+        score = fmaf(e1, c.w, score);
+        if (MODE == 0) {
+          abar[OFF + x] += e0;
+          abar[OFF + x + 1] += e1;
+        } else {
+          plogp = fmaf(e0, fmaf(t0, kLn2, p.ln_hq), plogp);
+          plogp = fmaf(e1, fmaf(t1, kLn2, p.ln_hq), plogp);
+        }
       }
     }
-    __device__ __forceinline__ void chunk_text(const Params& p, const uint32_t (&r)[32], const float2* c2) {
+    __device__ __forceinline__ void chunk_text(const Params& p, const uint32_t (&r)[32], const float4* c4) {
 #pragma unroll
-      for (int x = 0; x < 32; ++x) {
-        const float2 c = c2[x];
+      for (int x = 0; x < 32; x += 2) {
+        const float4 c = c4[x / 2];
         score = fmaf(fast_exp2(fmaf(__uint_as_float(r[x]), p.sc2, -c.x)), c.y, score);
+        score = fmaf(fast_exp2(fmaf(__uint_as_float(r[x + 1]), p.sc2, -c.z)), c.w, score);
       }
     }
     // `masked`: some key of the warp lies inside the observation window (the last W of the sequence), so
     // window rows before first_row do not see it.  Those logits are replaced by a hugely negative
     // value, whose exp2 is exactly zero, and the ordinary routines run.  Only the last key block
     // gets here.
-    __device__ __forceinline__ void chunk(const Params& p, uint32_t (&r)[32], int local, int md, int first_row,
-                                          bool masked) {
+    __device__ __forceinline__ void chunk(const Params& p, uint32_t (&r)[32], int local) {
       if (masked) {
         const int row0 = local % W;
 #pragma unroll
         for (int x = 0; x < 32; ++x) if (row0 + x < first_row) r[x] = __float_as_uint(-1e30f);
       }
       if (md == MEDA_VISUAL) {
-        if (W == 32 || local % W == 0) chunk_visual<0>(p, r, cvis + local);
-        else chunk_visual<(W > 32 ? 32 : 0)>(p, r, cvis + local);
+        if (W == 32 || local % W == 0) chunk_visual<0>(p, r, cvis + local / 2);
+        else chunk_visual<(W > 32 ? 32 : 0)>(p, r, cvis + local / 2);
       } else {
-        chunk_text(p, r, ctext + local);
+        chunk_text(p, r, ctext + local / 2);
       }
     }
     __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
-      const int j = it.a_row + row_in_block;               // this thread's key
-      const bool valid = j < p.n;
-      const int md = p.modality[j];                        // the padded map covers j up to the block end
-      const int first_row = j - (p.n - W);                 // causal: window rows i >= first_row see key j
-      const bool masked = __any_sync(0xffffffffu, valid && first_row > 0);
       const int n_chunks = (tile == it.n_tiles - 1 ? it.last_n : 128) / 32;
-      const int local0 = tile * 128;
+      const int local0 = tile * 128;                       // column inside the KV group: head * W + row
       // two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced
       uint32_t ra[32], rb[32];
       sm100::tmem_ld_32x32_issue(taddr, ra);
       sm100::tmem_ld_wait();
       sm100::tmem_ld_pin(ra);
       if (n_chunks > 1) sm100::tmem_ld_32x32_issue(taddr + 32u, rb);
-      if (valid) chunk(p, ra, local0, md, first_row, masked);
+      if (valid) chunk(p, ra, local0);
       if (n_chunks > 1) {
         sm100::tmem_ld_wait();
         sm100::tmem_ld_pin(rb);
         if (n_chunks > 2) sm100::tmem_ld_32x32_issue(taddr + 64u, ra);
-        if (valid) chunk(p, rb, local0 + 32, md, first_row, masked);
+        if (valid) chunk(p, rb, local0 + 32);
       }
       if (n_chunks > 2) {
         sm100::tmem_ld_wait();
         sm100::tmem_ld_pin(ra);
         if (n_chunks > 3) sm100::tmem_ld_32x32_issue(taddr + 96u, rb);
-        if (valid) chunk(p, ra, local0 + 64, md, first_row, masked);
+        if (valid) chunk(p, ra, local0 + 64);
       }
       if (n_chunks > 3) {
         sm100::tmem_ld_wait();
         sm100::tmem_ld_pin(rb);
-        if (valid) chunk(p, rb, local0 + 96, md, first_row, masked);
+        if (valid) chunk(p, rb, local0 + 96);
       }
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {

@@ -246,6 +246,7 @@ void launch_sweep_policy(meda_ctx* ctx, const CUtensorMap& map_k, const CUtensor
   prm.n = c.n_tokens; prm.hkv = c.n_kv_heads; prm.cols = ctx->group * c.window;
   prm.n_blocks = (c.n_tokens + 255) / 256;
   prm.sc2 = kLog2e / sqrtf((float)c.head_dim);
+  prm.ln_hq = logf((float)c.n_q_heads);
   umma_stream_kernel<Policy><<<std::min(prm.n_blocks, ctx->sm_count), us_threads<Policy>(), StreamShared<Policy>::alloc, st>>>(
       map_k, map_q, prm, ctx->ws.status);
 }
@@ -268,7 +269,7 @@ meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, c
   {
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
     sweep_coef_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_stats, ctx->ws.coef_vis, ctx->ws.coef_text, rows,
-                                                          1.0f / (float)c.n_q_heads);
+                                                          (float)c.n_q_heads);
   }
   {
     LaunchScope scope(ctx, MEDA_K_SWEEP, st);

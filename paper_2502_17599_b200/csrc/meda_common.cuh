@@ -18,7 +18,7 @@ constexpr float kCosEps = 1e-8f;      // lower clamp of a key norm (Eq. 11 is si
 
 struct Workspace {
   uint8_t* modality = nullptr;        // [n padded to a multiple of 256, + 128] 0 = text, 1 = visual, 2 = padding
-  float4* coef_vis = nullptr;         // [Hq * w] per-column constants of the tensor-core scores sweep
+  float2* coef_vis = nullptr;         // [Hq * w] per-column constants of the tensor-core scores sweep
   float2* coef_text = nullptr;        // [Hq * w]
   int* status = nullptr;              // device status word (first error wins)
   float* stats_partial = nullptr;     // [chunks][Hq][w][4]

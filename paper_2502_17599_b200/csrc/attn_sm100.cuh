@@ -138,24 +138,18 @@ struct StatsPolicy {
       reinterpret_cast<uint32_t*>(mod_t)[lane] = __ldg(reinterpret_cast<const uint32_t*>(p.modality + c0) + lane);
       __syncwarp();
       if (!__any_sync(0xffffffffu, valid)) return;
-      // two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced
-      uint32_t ra[32], rb2[32];
-      sm100::tmem_ld_32x32_issue(taddr, ra);
-      sm100::tmem_ld_wait();
-      sm100::tmem_ld_pin(ra);
-      sm100::tmem_ld_32x32_issue(taddr + 32u, rb2);
-      if (valid) chunk(p, ra, 0, c0, last_visible);
-      sm100::tmem_ld_wait();
-      sm100::tmem_ld_pin(rb2);
-      sm100::tmem_ld_32x32_issue(taddr + 64u, ra);
-      if (valid) chunk(p, rb2, 1, c0 + 32, last_visible);
-      sm100::tmem_ld_wait();
-      sm100::tmem_ld_pin(ra);
-      sm100::tmem_ld_32x32_issue(taddr + 96u, rb2);
-      if (valid) chunk(p, ra, 2, c0 + 64, last_visible);
-      sm100::tmem_ld_wait();
-      sm100::tmem_ld_pin(rb2);
-      if (valid) chunk(p, rb2, 3, c0 + 96, last_visible);
+      // One chunk in registers at a time: with four epilogue warps per scheduler the load latency hides
+      // behind the other warps, and a second buffer does not fit the 96 registers a 576-thread block
+      // leaves (a kernel with a tensor-memory load in flight must not spill: the destination
+      // registers could be saved before the load has landed).
+      uint32_t acc[32];
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        sm100::tmem_ld_32x32_issue(taddr + 32u * c, acc);
+        sm100::tmem_ld_wait();
+        sm100::tmem_ld_pin(acc);
+        if (valid) chunk(p, acc, c, c0 + 32 * c, last_visible);
+      }
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {
       const int g = it.u0 >> 16, rb = it.u0 & 65535;
@@ -326,6 +320,19 @@ struct SweepPolicy {
     __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
       const int n_chunks = (tile == it.n_tiles - 1 ? it.last_n : 128) / 32;
       const int local0 = tile * 128;                       // column inside the KV group: head * W + row
+      if (W > 32) {
+        // 64 running sums per thread leave no room for a second register buffer (nothing may spill
+        // while a tensor-memory load is in flight): one chunk at a time
+        uint32_t acc[32];
+#pragma unroll 1
+        for (int c = 0; c < n_chunks; ++c) {
+          sm100::tmem_ld_32x32_issue(taddr + 32u * c, acc);
+          sm100::tmem_ld_wait();
+          sm100::tmem_ld_pin(acc);
+          if (valid) chunk(p, acc, local0 + 32 * c);
+        }
+        return;
+      }
       // two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced
       uint32_t ra[32], rb[32];
       sm100::tmem_ld_32x32_issue(taddr, ra);

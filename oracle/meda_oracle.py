@@ -411,6 +411,29 @@ def compress_pass(layers, modality: np.ndarray, global_budget: int, min_budget: 
 
 
 # --------------------------------------------------------------------------------------
+# After the pass: one decoding step over a (compressed) cache, Eq. 3
+# --------------------------------------------------------------------------------------
+
+def decode_attention(q: np.ndarray, k_c: np.ndarray, v_c: np.ndarray) -> np.ndarray:
+    """Attention of one new token's queries over a per-layer cache (Eq. 3): for every query head h of
+    KV group g, out[h] = softmax(q_h K_g^T / sqrt(d)) V_g over all rows of the cache (the new token
+    comes after every cached one, so nothing is masked).  The cache may be the full one or the
+    compressed (K_c, V_c) of Eq. 10 / Eq. 12; merged rows are used as they are, with no weighting by
+    how many pairs they absorbed (Eq. 3 has none).  q [Hq, d], k_c, v_c [Hkv, S, d] -> [Hq, d]."""
+    hq, d = q.shape
+    hkv = k_c.shape[0]
+    group = hq // hkv
+    out = np.zeros((hq, d))
+    for h in range(hq):
+        g = h // group
+        s = (k_c[g] @ q[h]) / np.sqrt(float(d))
+        p = np.exp(s - s.max())
+        p /= p.sum()
+        out[h] = p @ v_c[g]
+    return out
+
+
+# --------------------------------------------------------------------------------------
 # Off the hot path: the appendix's KV-cache memory formula (context for Table 6)
 # --------------------------------------------------------------------------------------
 

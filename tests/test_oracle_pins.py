@@ -426,3 +426,29 @@ def test_table6_headlines_and_memory_formula():
     assert O.kv_cache_gib(1) * 1024 == 0.5
     tokens_full = full[2] / O.kv_cache_gib(1)
     assert 4900 < tokens_full < 5000
+
+
+def test_decode_attention_closed_forms_and_bruteforce():
+    """Eq. 3: zero query = mean of the values; a key aligned with the query and scaled up = that row's
+    value; adding a constant vector to every key changes nothing; brute-force loops on a small case."""
+    rng = np.random.default_rng(21)
+    hq, hkv, s_rows, d = 6, 2, 37, 16
+    q = rng.normal(size=(hq, d))
+    k = rng.normal(size=(hkv, s_rows, d))
+    v = rng.normal(size=(hkv, s_rows, d))
+    np.testing.assert_allclose(O.decode_attention(np.zeros_like(q), k, v), np.repeat(v.mean(axis=1), hq // hkv, axis=0), atol=1e-12)
+    k2 = k.copy()
+    k2[1, 5] = 400.0 * q[4] / np.linalg.norm(q[4])           # head 4 belongs to KV group 1
+    np.testing.assert_allclose(O.decode_attention(q, k2, v)[4], v[1, 5], atol=1e-9)
+    np.testing.assert_allclose(O.decode_attention(q, k + rng.normal(size=(1, 1, d)), v), O.decode_attention(q, k, v), atol=1e-10)
+    want = np.zeros((hq, d))
+    for h in range(hq):
+        g = h // (hq // hkv)
+        logits = [sum(q[h][t] * k[g][j][t] for t in range(d)) / math.sqrt(d) for j in range(s_rows)]
+        m = max(logits)
+        w = [math.exp(x - m) for x in logits]
+        z = sum(w)
+        for t in range(d):
+            want[h][t] = sum(w[j] * v[g][j][t] for j in range(s_rows)) / z
+    np.testing.assert_allclose(O.decode_attention(q, k, v), want, atol=1e-12)
+

@@ -40,6 +40,7 @@ def parse_args():
     ap.add_argument("--eager", action="store_true", help="time eager launches instead of a CUDA-graph replay of the pass")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="skip the decoding-step context measurement")
     ap.add_argument("--e2e-steps", type=int, default=2)
     return ap.parse_args()
 
@@ -319,6 +320,44 @@ def run_ours(args):
     ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
     value = whole_job_throughput(wl, world, ms_step)
 
+    # context: one decoding step's attention (Eq. 3) over all layers, compressed caches against full ones
+    decode = None
+    if not args.no_decode and wl.head_dim in (64, 128) and (wl.n_q_heads // wl.n_kv_heads) in (1, 2, 3, 4, 7, 8):
+        q_new = [q_[:, -1, :].contiguous() for q_ in qs]
+        out = torch.zeros((wl.n_q_heads, wl.head_dim), dtype=torch.float32, device="cuda")
+
+        def decode_ms(compressed):
+            def one():
+                for l in range(L):
+                    if compressed:
+                        cp.ctx.decode_attention(l, q_new[l], cp.k_out[l], cp.v_out[l], out, budgets=cp.budgets)
+                    else:
+                        cp.ctx.decode_attention(l, q_new[l], ks[l], vs[l], out, n_rows=wl.n_tokens)
+            one()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                one()
+            for _ in range(3):
+                graph.replay()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(10):
+                graph.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / 10
+
+        ms_c, ms_f = decode_ms(True), decode_ms(False)
+        e = wl.element_size
+        bytes_c = 2 * wl.n_kv_heads * wl.head_dim * e * float(budgets.sum())
+        bytes_f = 2 * wl.n_kv_heads * wl.head_dim * e * float(L * wl.n_tokens)
+        decode = {"what": "attention of one new token over every layer's cache (Eq. 3), one CUDA-graph replay per token",
+                  "ms_per_token_compressed": ms_c, "ms_per_token_full": ms_f, "speedup": ms_f / ms_c,
+                  "cache_bytes_compressed": bytes_c, "cache_bytes_full": bytes_f,
+                  "GB/s_compressed": bytes_c / ms_c / 1e6, "GB/s_full": bytes_f / ms_f / 1e6}
+        cp.check()
+
     # end-to-end leg: pinned host inputs -> device -> pass -> compacted caches back to the host
     e2e = None
     if not args.no_e2e:
@@ -407,7 +446,7 @@ def run_ours(args):
                              + f", layers alternate between {len(cp.contexts)} streams"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roof, "kernels": per_class, "kernel_rooflines": extra, "cpu_baseline": cpu,
-        "budgets_min_max": [int(budgets.min()), int(budgets.max())],
+        "budgets_min_max": [int(budgets.min()), int(budgets.max())], "decode_context": decode,
     }
     print(json.dumps(out), flush=True)
     if world > 1:

@@ -164,6 +164,20 @@ meda_status meda_compress_layer(meda_ctx* ctx, int32_t layer, const void* k, con
                                 const int32_t* budgets, void* k_out, void* v_out, int32_t* counts,
                                 int32_t* idx_conserved, int32_t out_capacity, void* stream);
 
+/* After the pass: attention of one new token's queries over one layer's cache (Eq. 3), the step the compressed
+ * caches exist for.  out[h] = softmax(q_h . K_g^T / sqrt(head_dim)) V_g over the cache's rows, g the KV head of
+ * query head h; the new token comes after every cached one, so nothing is masked, and merged rows are used as
+ * they are (Eq. 3 carries no weights).
+ *   q        device, `dtype`, [n_q_heads][head_dim]
+ *   k_cache, v_cache  device, `dtype`, [n_kv_heads][capacity][head_dim]: the k_out / v_out of this layer, or a
+ *            full cache
+ *   budgets  device int32 [n_layers][3] or NULL.  Not NULL: the row count is S_layer, read on the device.
+ *            NULL: the row count is n_rows (1 <= n_rows <= capacity), for a cache that was not compressed.
+ *   out      device fp32 [n_q_heads][head_dim]
+ * Supported: head_dim 64 or 128, n_q_heads / n_kv_heads in {1, 2, 3, 4, 7, 8}; otherwise MEDA_ERR_UNSUPPORTED. */
+meda_status meda_decode_attention(meda_ctx* ctx, int32_t layer, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* budgets, int32_t n_rows, int32_t capacity, float* out, void* stream);
+
 /* ---- entry point that allocates nothing (the paper has no counterpart) ---------------------- */
 
 /* Largest n_q_heads * window the entry point below accepts, and the size of the scratch array
@@ -217,6 +231,7 @@ enum {
   MEDA_K_NEAREST,        /* similarity contraction + arg-max */
   MEDA_K_GROUP,          /* grouping of the less-important rows by target slot */
   MEDA_K_REDUCE,         /* segmented average */
+  MEDA_K_DECODE,         /* decoding-step attention over a cache */
   MEDA_K_CLASSES
 };
 

@@ -24,7 +24,7 @@ MEDA_ERR_CUDA = -5
 MEDA_ERR_UNSUPPORTED = -6
 MEDA_ERR_TIMEOUT = -7
 
-N_KERNEL_CLASSES = 10
+N_KERNEL_CLASSES = 11
 
 MEDA_BF16 = 0
 MEDA_F32 = 1
@@ -67,6 +67,8 @@ EXPORTS = {
     "meda_window_scores": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
     "meda_layer_entropy": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 5 +
                            [ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]),
+    "meda_decode_attention": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
+                              [ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]),
     "meda_row_stats_static": (ctypes.c_int, [ctypes.c_void_p] * 3 + [ctypes.c_int32] * 6 + [ctypes.c_void_p] * 2),
     "meda_allocate_budgets": (ctypes.c_int, [ctypes.c_void_p] * 4),
     "meda_select_topk": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
@@ -226,3 +228,9 @@ class Context:
         _check(self._lib.meda_compress_layer(self._h, layer, _ptr(k), _ptr(v), _ptr(scores), _ptr(budgets),
                                              _ptr(k_out), _ptr(v_out), _ptr(counts), _ptr(idx_conserved),
                                              out_capacity, _stream(stream)), "meda_compress_layer")
+
+    def decode_attention(self, layer, q, k_cache, v_cache, out, budgets=None, n_rows=0, capacity=None, stream=None):
+        cap = k_cache.shape[1] if capacity is None else capacity
+        _check(self._lib.meda_decode_attention(self._h, layer, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(budgets),
+                                               int(n_rows), int(cap), _ptr(out), _stream(stream)), "meda_decode_attention")
+

@@ -12,6 +12,7 @@
 #include "allocate.cuh"
 #include "attn_generic.cuh"
 #include "attn_sm100.cuh"
+#include "decode.cuh"
 #include "meda_common.cuh"
 #include "group_reduce.cuh"
 #include "merge_generic.cuh"
@@ -47,6 +48,7 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.modality);
   cudaFree(ws.status);
   cudaFree(ws.stats_partial);
+  cudaFree(ws.decode_partial);
   cudaFree(ws.row_stats_vis);
   cudaFree(ws.ent_partial);
   cudaFree(ws.inv_norm);
@@ -487,10 +489,56 @@ meda_status static_stats_scratch(float** partial) {
   return MEDA_OK;
 }
 
+// ---- decoding step over a layer's cache --------------------------------------------------------
+template <typename T, int D, int G>
+meda_status launch_decode_g(meda_ctx* ctx, const void* q, const void* k_c, const void* v_c, const int32_t* budget_row,
+                            int rows, int cap, float* out, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  {
+    LaunchScope scope(ctx, MEDA_K_DECODE, st);
+    decode_partial_kernel<T, D, G><<<dim3(kDecSplits, c.n_kv_heads), kDecWarps * 32, 0, st>>>(
+        static_cast<const T*>(q), static_cast<const T*>(k_c), static_cast<const T*>(v_c), budget_row, rows, cap,
+        ctx->ws.decode_partial, 1.0f / sqrtf((float)D));
+  }
+  LaunchScope scope(ctx, MEDA_K_DECODE, st);
+  decode_combine_kernel<D><<<c.n_q_heads, D, 0, st>>>(ctx->ws.decode_partial, budget_row, rows, cap, out);
+  return launch_status();
+}
+
+template <typename T, int D>
+meda_status launch_decode(meda_ctx* ctx, const void* q, const void* k_c, const void* v_c, const int32_t* budget_row,
+                          int rows, int cap, float* out, cudaStream_t st) {
+  switch (ctx->group) {
+    case 1: return launch_decode_g<T, D, 1>(ctx, q, k_c, v_c, budget_row, rows, cap, out, st);
+    case 2: return launch_decode_g<T, D, 2>(ctx, q, k_c, v_c, budget_row, rows, cap, out, st);
+    case 3: return launch_decode_g<T, D, 3>(ctx, q, k_c, v_c, budget_row, rows, cap, out, st);
+    case 4: return launch_decode_g<T, D, 4>(ctx, q, k_c, v_c, budget_row, rows, cap, out, st);
+    case 7: return launch_decode_g<T, D, 7>(ctx, q, k_c, v_c, budget_row, rows, cap, out, st);
+    case 8: return launch_decode_g<T, D, 8>(ctx, q, k_c, v_c, budget_row, rows, cap, out, st);
+    default: return MEDA_ERR_UNSUPPORTED;
+  }
+}
+
 }  // namespace
 
 #pragma GCC visibility push(default)
 extern "C" {
+
+meda_status meda_decode_attention(meda_ctx* ctx, int32_t layer, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* budgets, int32_t n_rows, int32_t capacity, float* out, void* stream) {
+  if (!layer_ok(ctx, layer) || !q || !k_cache || !v_cache || !out) return MEDA_ERR_INVALID_ARG;
+  if (capacity < 1 || (!budgets && (n_rows < 1 || n_rows > capacity))) return MEDA_ERR_INVALID_ARG;
+  const meda_config& c = ctx->cfg;
+  const int32_t* row = budgets ? budgets + (size_t)layer * 3 : nullptr;
+  cudaStream_t st = as_stream(stream);
+  if (c.head_dim == 64)
+    return c.dtype == MEDA_F32 ? launch_decode<float, 64>(ctx, q, k_cache, v_cache, row, n_rows, capacity, out, st)
+                               : launch_decode<__nv_bfloat16, 64>(ctx, q, k_cache, v_cache, row, n_rows, capacity, out, st);
+  if (c.head_dim == 128)
+    return c.dtype == MEDA_F32 ? launch_decode<float, 128>(ctx, q, k_cache, v_cache, row, n_rows, capacity, out, st)
+                               : launch_decode<__nv_bfloat16, 128>(ctx, q, k_cache, v_cache, row, n_rows, capacity, out, st);
+  return MEDA_ERR_UNSUPPORTED;
+}
 
 meda_status meda_row_stats_static(const void* q_win, const void* k, const uint8_t* modality, int32_t n_q_heads,
                                   int32_t n_kv_heads, int32_t head_dim, int32_t n_tokens, int32_t window,
@@ -620,6 +668,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     if (st == MEDA_OK) st = raise_sweep_smem<64, 1>();
   }
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
+  if (st == MEDA_OK) st = carve(&ws.decode_partial, (int64_t)c.n_q_heads * kDecSplits * (c.head_dim + 2), &ws.bytes);
   ctx->sort_chunks = (int)((n + kSortBlockItems - 1) / kSortBlockItems + 7) / 8 * 8;   // padded: the scan works on whole vectors
   ctx->seg_chunks = (int)((n + kSegChunk - 1) / kSegChunk);
   ctx->sort_passes = n <= kSortBins ? 1 : (n <= (int64_t)kSortBins * kSortBins ? 2 : 3);
@@ -683,7 +732,7 @@ int64_t meda_launch_count(const meda_ctx* ctx) { return ctx ? ctx->launches : 0;
 
 const char* meda_kernel_class_name(int32_t kernel_class) {
   static const char* const names[MEDA_K_CLASSES] = {"stats", "stats_combine", "sweep", "entropy_final", "allocate",
-                                                    "select", "prep", "nearest", "group", "reduce"};
+                                                    "select", "prep", "nearest", "group", "reduce", "decode"};
   return kernel_class >= 0 && kernel_class < MEDA_K_CLASSES ? names[kernel_class] : nullptr;
 }
 

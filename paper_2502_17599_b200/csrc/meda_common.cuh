@@ -24,6 +24,7 @@ struct Workspace {
   float* stats_partial = nullptr;     // [chunks][Hq][w][4]
   float* row_stats_vis = nullptr;     // [Hq][<= kMaxWindow][4] normalisers of the visual query window (E_VT)
   float* ent_partial = nullptr;       // [ent_slots]
+  float* decode_partial = nullptr;    // [Hq][splits][d + 2] partial softmax states of the decoding step
   float* inv_norm = nullptr;          // [Hkv][inv_stride]  1 / max(|k_c|, eps) per conserved slot
   __nv_bfloat16* kc = nullptr;        // [Hkv][kc_rows][128] gathered conserved keys (bf16, head_dim 128 only)
   int32_t* sort_keys[2] = {nullptr, nullptr};   // [Hkv][n] ping-pong: target slot of each sorted entry

@@ -344,3 +344,31 @@ def test_cross_modal_entropy_with_the_vision_to_text_term(wl, entropy_mode):
         assert float(buf.entropy[l]) == float(both[l])
     ctx.close()
 
+
+
+@pytest.mark.parametrize("wl", small_cases(), ids=lambda w: w.name)
+def test_decode_attention_over_compressed_and_full_caches(wl):
+    """Eq. 3 on the device: one new token's queries over the compacted cache of a layer (row count read
+    from the budgets on the device) and over the full cache (row count given)."""
+    group = wl.n_q_heads // wl.n_kv_heads
+    if group not in (1, 2, 3, 4, 7, 8) or wl.head_dim not in (64, 128):
+        pytest.skip("shape outside the decoding kernel's list")
+    ctx = make_ctx(wl)
+    buf = P.GpuBuffers(wl)
+    n = wl.n_tokens
+    (q, k, v), (qh, kh, vh) = P.layer_inputs(wl, 0, "cuda")
+    ctx.window_scores(0, q, k, buf.row_stats, buf.scores, buf.entropy)
+    S = max(wl.window, n // 5)
+    M = (3 * S) // 4
+    budgets = torch.tensor([[S, M, S - M]] * wl.n_layers, dtype=torch.int32, device="cuda")
+    ctx.compress_layer(0, k, v, buf.scores, budgets, buf.k_out, buf.v_out, buf.counts, buf.idx_c, buf.cap)
+    q_new = q[:, -1, :].contiguous()                       # the last window row stands in for the new token's query
+    out = torch.zeros((wl.n_q_heads, wl.head_dim), dtype=torch.float32, device="cuda")
+    ctx.decode_attention(0, q_new, buf.k_out, buf.v_out, out, budgets=budgets)
+    ctx.check()
+    want = O.decode_attention(P.np64(q_new), P.np64(buf.k_out[:, :S]), P.np64(buf.v_out[:, :S]))
+    np.testing.assert_allclose(P.np64(out), want, rtol=1e-4, atol=1e-4)
+    ctx.decode_attention(0, q_new, k, v, out, n_rows=n)
+    ctx.check()
+    np.testing.assert_allclose(P.np64(out), O.decode_attention(P.np64(q_new), kh, vh), rtol=1e-4, atol=1e-4)
+    ctx.close()

@@ -111,9 +111,27 @@ struct NearestRow {
     const float u2 = sm100::fmax3(t[6], t[7], t[8]), u3 = sm100::fmax3(t[9], t[10], t[11]);
     const float cmax = fmaxf(sm100::fmax3(u0, u1, u2), u3);
     if (cmax > best) {
-      int first = 31;
+      // First slot that attains the maximum.  The four sub-maxima of the reduction tree say which
+      // nine-column group holds it, so only that group is scanned; the few lanes that improve in a
+      // chunk rarely sit in more than one or two groups, which is what the warp pays for.
+      int first;
+      if (u0 == cmax) {
+        first = 8;
 #pragma unroll
-      for (int x = 30; x >= 0; --x) if (v[x] == cmax) first = x;
+        for (int x = 7; x >= 0; --x) if (v[x] == cmax) first = x;
+      } else if (u1 == cmax) {
+        first = 17;
+#pragma unroll
+        for (int x = 16; x >= 9; --x) if (v[x] == cmax) first = x;
+      } else if (u2 == cmax) {
+        first = 26;
+#pragma unroll
+        for (int x = 25; x >= 18; --x) if (v[x] == cmax) first = x;
+      } else {
+        first = 31;
+#pragma unroll
+        for (int x = 30; x >= 27; --x) if (v[x] == cmax) first = x;
+      }
       best = cmax;
       best_slot = s0 + first;
     }

@@ -65,11 +65,14 @@ class CompressionPass:
             ev.record(s)
             main.wait_event(ev)
 
-    def run(self, q_layers, k_layers, v_layers, stream=None, single_stream=False):
+    def run(self, q_layers, k_layers, v_layers, stream=None, single_stream=False, qk_ready=None, v_ready=None):
         """Enqueues the whole pass.  Inputs are lists of per-layer device tensors; results stay on the
         device in this object's buffers.  The work is ordered after what `stream` (default: torch's
         current stream) holds and `stream` waits for all of it.  With `single_stream` everything goes to
-        `stream` through the first context (used when every launch is timed on its own)."""
+        `stream` through the first context (used when every launch is timed on its own).  `qk_ready` /
+        `v_ready`: optional per-layer events after which a layer's (queries, keys) / values are in
+        place (copies still in flight on another stream): phase A of a layer waits for the first,
+        phase B for the second."""
         L = self.wl.n_layers
         main = stream if stream is not None else torch.cuda.current_stream()
         if single_stream or not self.streams:
@@ -79,6 +82,8 @@ class CompressionPass:
             self._fork(main)
         for l in range(L):
             c, s, rs = lanes[l % len(lanes)]
+            if qk_ready is not None:
+                s.wait_event(qk_ready[l])
             c.window_scores(l, q_layers[l], k_layers[l], rs, self.scores[l], self.entropy, s)
         if len(lanes) > 1:
             self._join(main)
@@ -87,6 +92,8 @@ class CompressionPass:
             self._fork(main)
         for l in range(L):
             c, s, _ = lanes[l % len(lanes)]
+            if v_ready is not None:
+                s.wait_event(v_ready[l])
             c.compress_layer(l, k_layers[l], v_layers[l], self.scores[l], self.budgets, self.k_out[l], self.v_out[l],
                              self.counts[l], self.idx_c[l], self.cap, s)
         if len(lanes) > 1:
@@ -118,11 +125,30 @@ class CompressionPass:
         head (see `alloc_host_outputs`).  Returns (h2d_bytes, d2h_bytes)."""
         L = self.wl.n_layers
         h2d = 0
-        for l in range(L):
-            for src, dst in ((q_host[l], staging["q"][l]), (k_host[l], staging["k"][l]), (v_host[l], staging["v"][l])):
-                dst.copy_(src, non_blocking=True)
-                h2d += src.numel() * src.element_size()
-        self.run(staging["q"], staging["k"], staging["v"])
+        # Copies run on their own stream, queries and keys of every layer first (phase A needs only
+        # those), then the values; each layer's kernels wait for that layer's copies only, so the pass
+        # overlaps with the transfer instead of following it.
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_copy_stream"):
+            self._copy_stream = torch.cuda.Stream(device=self.device)
+        cs = self._copy_stream
+        cs.wait_stream(main)
+        qk_ready, v_ready = [], []
+        with torch.cuda.stream(cs):
+            for l in range(L):
+                for src, dst in ((q_host[l], staging["q"][l]), (k_host[l], staging["k"][l])):
+                    dst.copy_(src, non_blocking=True)
+                    h2d += src.numel() * src.element_size()
+                ev = torch.cuda.Event()
+                ev.record(cs)
+                qk_ready.append(ev)
+            for l in range(L):
+                staging["v"][l].copy_(v_host[l], non_blocking=True)
+                h2d += v_host[l].numel() * v_host[l].element_size()
+                ev = torch.cuda.Event()
+                ev.record(cs)
+                v_ready.append(ev)
+        self.run(staging["q"], staging["k"], staging["v"], qk_ready=qk_ready, v_ready=v_ready)
         out_host["budgets"].copy_(self.budgets, non_blocking=True)
         torch.cuda.current_stream().synchronize()      # the live row counts decide what comes back
         d2h = self.budgets.numel() * 4

@@ -208,11 +208,11 @@ def algorithmic_work(wl, budgets):
 
 # DRAM traffic of one launch of the arg-max kernel, dram__bytes_read.sum + dram__bytes_write.sum from the
 # ncu capture summarised in profiles/hot_kernels_long_video_128k_first2layers.md (134.3 MB read: the key
-# cache once, whatever the budget, plus the gathered keys; 4.6 MB written).  It is reported only while
+# cache once, whatever the budget, plus the gathered keys; 4.5 MB written).  It is reported only while
 # the kernel's sources still hash to what was captured.
-NEAREST_TRAFFIC_BYTES = 138.9e6
+NEAREST_TRAFFIC_BYTES = 138.8e6
 NEAREST_SOURCES = ("paper_2502_17599_b200/csrc/nearest_sm100.cuh", "paper_2502_17599_b200/csrc/sm100_primitives.cuh")
-NEAREST_SOURCES_SHA = "69a1b0a6fffe1d3c"
+NEAREST_SOURCES_SHA = "608d0aaf608faca7"
 
 
 def nearest_traffic():

@@ -372,3 +372,41 @@ def test_decode_attention_over_compressed_and_full_caches(wl):
     ctx.check()
     np.testing.assert_allclose(P.np64(out), O.decode_attention(P.np64(q_new), kh, vh), rtol=1e-4, atol=1e-4)
     ctx.close()
+
+
+def test_degenerate_sizes_on_the_tensor_core_paths():
+    """A prompt shorter than one tile (n = 97 < 128 keys, one ragged tile everywhere), and budgets at both
+    ends: every token conserved (nothing to merge: outputs are the inputs) and the smallest budget."""
+    n = 97
+    wl = W.small_variant("short_prompt", spans=((0, 11, 0), (11, 70, 1), (70, 97, 0)), window=32, frame_tokens=0,
+                         salient_frac=0.0, rho=0.4, seed=9)
+    assert wl.n_tokens == n
+    ctx = make_ctx(wl)
+    buf = P.GpuBuffers(wl)
+    mod = wl.modality().numpy()
+    (q, k, v), (qh, kh, vh) = P.layer_inputs(wl, 0, "cuda")
+    ctx.window_scores(0, q, k, buf.row_stats, buf.scores, buf.entropy)
+    ctx.check()
+    P.assert_scores_close(P.np64(buf.scores), O.window_scores(qh, kh))
+    P.assert_entropy_close(float(buf.entropy[0]), O.cross_modal_entropy(qh, kh, mod))
+    a_s = P.np64(buf.scores)
+    for S in (n, wl.window, 1):
+        M = (3 * S) // 4
+        budgets = torch.tensor([[S, M, S - M]] * wl.n_layers, dtype=torch.int32, device="cuda")
+        buf.k_out.fill_(7.0)
+        ctx.select_topk(0, buf.scores, budgets, buf.idx_c, buf.idx_less, buf.cap)
+        ctx.merge_kv(0, k, v, budgets, buf.idx_c, buf.idx_less, buf.k_out, buf.v_out, buf.counts, buf.target, buf.cap)
+        ctx.check()
+        for g in range(wl.n_kv_heads):
+            cons = buf.idx_c[g, :S].cpu().numpy().astype(np.int64)
+            less = buf.idx_less[g, : n - S].cpu().numpy().astype(np.int64)
+            assert P.compare_selection(cons, a_s[g], mod, M, S - M) == 0
+            tgt = buf.target[g, : n - S].cpu().numpy()
+            P.compare_targets(tgt, kh[g], cons, less)
+            P.compare_merged(P.np64(buf.k_out[g, :S]), P.np64(buf.v_out[g, :S]), buf.counts[g, :S].cpu().numpy(),
+                             kh[g], vh[g], cons, less, tgt, wl.dtype)
+            assert int(buf.counts[g, :S].sum()) == n
+        if S == n:
+            assert torch.equal(buf.k_out[:, :n], k) and torch.equal(buf.v_out[:, :n], v) and (buf.counts[:, :n] == 1).all()
+        assert (buf.k_out[:, S:] == 7.0).all()
+    ctx.close()

@@ -1,5 +1,5 @@
 #!/usr/bin/env python
-"""Benchmark of the MEDA compression pass (see the design doc for what is measured and how).
+"""Benchmark of the MEDA compression pass.
 
 One "step" = the whole pass (phase A of every layer, the budget barrier, phase B of every layer)
 over one synthetic prompt.  The metric is KV tokens compressed per second per layer-pass:
@@ -192,7 +192,9 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 
 def algorithmic_work(wl, budgets):
-    """Algorithmic bytes / flops per layer-pass of each kernel class ('Roofline')."""
+    """Algorithmic bytes / flops per layer-pass of each kernel class: stats reads the key cache once,
+    the sweep reads it once and writes the scores, the similarity contraction is 2 (n - S) S d flops per
+    head, the segmented average reads every key and value row once and writes the S merged rows."""
     e = wl.element_size
     n, d, hkv, hq, w = wl.n_tokens, wl.head_dim, wl.n_kv_heads, wl.n_q_heads, wl.window
     kbytes = hkv * n * d * e
@@ -207,7 +209,7 @@ def algorithmic_work(wl, budgets):
 
 
 # DRAM traffic of one launch of the arg-max kernel, dram__bytes_read.sum + dram__bytes_write.sum from the
-# ncu capture summarised in profiles/hot_kernels_long_video_128k_first2layers.md (134.3 MB read: the key
+# ncu capture whose summary is kept under profiles/ (134.3 MB read: the key
 # cache once, whatever the budget, plus the gathered keys; 4.5 MB written).  It is reported only while
 # the kernel's sources still hash to what was captured.
 NEAREST_TRAFFIC_BYTES = 138.8e6

@@ -49,7 +49,7 @@ typedef enum {
   MEDA_ERR_BUDGET_INFEASIBLE = -3, /* global budget outside [L*min_budget, L*n_tokens] */
   MEDA_ERR_WORKSPACE = -4,         /* an output capacity is too small for the layer's budget */
   MEDA_ERR_CUDA = -5,              /* a CUDA runtime call failed */
-  MEDA_ERR_UNSUPPORTED = -6,       /* valid request that this build does not implement */
+  MEDA_ERR_UNSUPPORTED = -6,       /* valid request that the library does not implement */
   MEDA_ERR_TIMEOUT = -7            /* a bounded device-side wait ran out */
 } meda_status;
 

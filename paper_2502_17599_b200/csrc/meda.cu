@@ -583,7 +583,7 @@ const char* meda_status_string(meda_status status) {
     case MEDA_ERR_BUDGET_INFEASIBLE: return "budget infeasible";
     case MEDA_ERR_WORKSPACE: return "output capacity too small";
     case MEDA_ERR_CUDA: return "CUDA runtime error";
-    case MEDA_ERR_UNSUPPORTED: return "not implemented in this build";
+    case MEDA_ERR_UNSUPPORTED: return "not implemented";
     case MEDA_ERR_TIMEOUT: return "bounded device wait ran out";
   }
   return "unknown status";

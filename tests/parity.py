@@ -1,7 +1,7 @@
 """Helpers shared by the GPU parity tests: running the CUDA path through the C-ABI binding,
 running the oracle on the same bits, and the comparison rules.
 
-Comparison rules (tolerances are the ones the task states):
+Comparison rules and tolerances:
   budgets          bit-exact
   selected sets    bit-exact except swaps between candidates whose ORACLE scores differ by less
                    than 1e-5 relative; swaps are counted and returned

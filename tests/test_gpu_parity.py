@@ -264,7 +264,7 @@ def test_end_to_end_with_teacher_forcing(wl):
         for g in range(wl.n_kv_heads):
             cons = buf.idx_c[g, :S].cpu().numpy().astype(np.int64)
             less = buf.idx_less[g, : n - S].cpu().numpy().astype(np.int64)
-            # selection is judged on the ORACLE's scores with the swap tolerance
+            # selection is compared on the ORACLE's scores with the swap tolerance
             swaps += P.compare_selection(cons, a_or[g], mod, M, N)
             np.testing.assert_array_equal(less, np.setdiff1d(np.arange(n), cons))
             tgt = buf.target[g, : n - S].cpu().numpy()

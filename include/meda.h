@@ -111,6 +111,14 @@ meda_status meda_poll_status(meda_ctx* ctx, void* stream);
 meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
                                float* row_stats, float* scores, float* entropy, void* stream);
 
+/* The second sweep of meda_window_scores alone, for a caller that already holds the window rows' softmax
+ * normalisers (for instance from the prefill attention kernel that produced the cache, if it also tracks the
+ * normaliser over the visual keys): one pass over the key cache instead of two.  row_stats is an INPUT here,
+ * fp32 [n_q_heads][window][4] with the layout and meaning meda_window_scores writes; scores and
+ * entropy[layer] (entropy may be NULL) are written exactly as by meda_window_scores. */
+meda_status meda_window_scores_from_stats(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                                          const float* row_stats, float* scores, float* entropy, void* stream);
+
 /* Cross-modal attention entropy of one layer (Eq. 4-6): E_CM = -(E_TV + E_VT), written to entropy[layer].
  *  - The E_TV term uses the text window q_win and its row_stats (from meda_window_scores): one sweep over
  *    the key cache, the same arithmetic as meda_window_scores' own entropy.  For callers that already hold

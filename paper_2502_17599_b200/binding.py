@@ -65,6 +65,7 @@ EXPORTS = {
     "meda_profile_read": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]),
     "meda_launch_count": (ctypes.c_int64, [ctypes.c_void_p]),
     "meda_window_scores": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
+    "meda_window_scores_from_stats": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
     "meda_layer_entropy": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 5 +
                            [ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]),
     "meda_decode_attention": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
@@ -203,6 +204,11 @@ class Context:
     def window_scores(self, layer, q_win, k, row_stats, scores, entropy=None, stream=None):
         _check(self._lib.meda_window_scores(self._h, layer, _ptr(q_win), _ptr(k), _ptr(row_stats), _ptr(scores),
                                             _ptr(entropy), _stream(stream)), "meda_window_scores")
+
+    def window_scores_from_stats(self, layer, q_win, k, row_stats, scores, entropy=None, stream=None):
+        _check(self._lib.meda_window_scores_from_stats(self._h, layer, _ptr(q_win), _ptr(k), _ptr(row_stats),
+                                                       _ptr(scores), _ptr(entropy), _stream(stream)),
+               "meda_window_scores_from_stats")
 
     def layer_entropy(self, layer, q_win, k, row_stats, entropy, q_vis=None, q_vis_pos=None, n_vis_rows=0, stream=None):
         _check(self._lib.meda_layer_entropy(self._h, layer, _ptr(q_win), _ptr(k), _ptr(row_stats), _ptr(q_vis),

@@ -805,6 +805,15 @@ meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, 
   return r;
 }
 
+meda_status meda_window_scores_from_stats(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
+                                          const float* row_stats, float* scores, float* entropy, void* stream) {
+  if (!layer_ok(ctx, layer) || !q_win || !k || !row_stats || !scores) return MEDA_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  if (ctx->fast_attn) return launch_sweep_fast(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+  if (ctx->cfg.dtype == MEDA_F32) return launch_sweep<float>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+  return launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+}
+
 meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
                                const void* q_vis, const int32_t* q_vis_pos, int32_t n_vis_rows, float* entropy,
                                void* stream) {

@@ -57,6 +57,11 @@ def test_phase_a_scores_stats_entropy(wl, entropy_mode):
         want_e = O.cross_modal_entropy(qh, kh, mod, entropy_mode=entropy_mode)
         P.assert_entropy_close(float(buf.entropy[l]), want_e)
         assert float(ent2[l]) == float(buf.entropy[l])      # the stand-alone sweep is the same arithmetic
+        # one sweep from given normalisers: the same bits as the two-sweep call
+        sc3, ent3 = torch.zeros_like(buf.scores), torch.zeros_like(buf.entropy)
+        ctx.window_scores_from_stats(l, q, k, buf.row_stats, sc3, ent3)
+        ctx.check()
+        assert torch.equal(sc3, buf.scores) and float(ent3[l]) == float(buf.entropy[l])
     ctx.close()
 
 

@@ -124,3 +124,58 @@ def test_full_size_pass_sampled_against_the_oracle(name):
                 assert ((err <= P.MERGE_BF16_ATOL) | (err <= ulp)).all(), (int(s), float(err.max()))
     print(f"{name}: layer {layer} (S={S}): tolerated selection swaps {swaps}, sampled arg-max near-ties {ties}")
     cp.close()
+
+
+def test_full_size_variants_ablation_modes_vision_to_text_term_and_decoding_step():
+    """The long-video 18.9K configuration at full size: the ablation modes of Table 5 (uniform budgets,
+    eviction instead of merging, mean of per-head entropies), the E_VT term with a window of visual query
+    rows, and one decoding step over the compressed cache of a layer, each against the oracle."""
+    from paper_2502_17599_b200.pipeline import CompressionPass
+    wl = W.WORKLOADS["long_video_19k"]
+    n, L, hkv = wl.n_tokens, wl.n_layers, wl.n_kv_heads
+    mod = wl.modality().numpy()
+    qs, ks, vs = [], [], []
+    for l in range(L):
+        q, k, v = W.make_layer(wl, l, "cuda")
+        qs.append(q); ks.append(k); vs.append(v)
+
+    # ---- "w/o dynamic allocation", "w/o merging", per-head entropies
+    cp = CompressionPass(wl, entropy_mode=1, alloc_mode=1, merge_mode=1)
+    cp.run(qs, ks, vs)
+    cp.check()
+    budgets = cp.budgets.cpu().numpy()
+    ent = P.np64(cp.entropy)
+    np.testing.assert_array_equal(budgets, O.allocate_budgets(ent, wl.global_budget, n, wl.min_budget, alloc_mode=1))
+    assert budgets[:, 0].max() - budgets[:, 0].min() <= 1 and int(budgets[:, 0].sum()) == wl.global_budget
+    layer = L // 2
+    qh = P.np64(qs[layer])
+    kh = np.stack([P.np64(ks[layer][g]) for g in range(hkv)])
+    P.assert_entropy_close(ent[layer], O.cross_modal_entropy(qh, kh, mod, entropy_mode=1))
+    S = int(budgets[layer, 0])
+    idx = cp.idx_c[layer, :, :S].long()
+    assert (cp.counts[layer, :, :S] == 1).all()
+    for g in range(hkv):
+        assert torch.equal(cp.k_out[layer, g, :S], ks[layer][g][idx[g]]) and torch.equal(cp.v_out[layer, g, :S], vs[layer][g][idx[g]])
+    cp.close()
+
+    # ---- the paper's modes: E_CM with the vision-to-text term, then one decoding step over the result
+    cp = CompressionPass(wl)
+    cp.run(qs, ks, vs)
+    cp.check()
+    n_rows = 32
+    qv, pos = W.make_visual_queries(wl, layer, n_rows, "cuda")
+    ent_full = cp.entropy.clone()
+    cp.ctx.layer_entropy(layer, None, ks[layer], None, ent_full, q_vis=qv, q_vis_pos=pos, n_vis_rows=n_rows)
+    cp.check()
+    want = O.cross_modal_entropy(qh, kh, mod, q_vis=P.np64(qv), q_vis_pos=pos.cpu().numpy().astype(np.int64))
+    P.assert_entropy_close(float(ent_full[layer]), want)
+    assert float(ent_full[layer]) > float(cp.entropy[layer])          # -E_VT is a positive addition
+
+    S = int(cp.budgets[layer, 0])
+    q_new = qs[layer][:, -1, :].contiguous()
+    out = torch.zeros((wl.n_q_heads, wl.head_dim), dtype=torch.float32, device="cuda")
+    cp.ctx.decode_attention(layer, q_new, cp.k_out[layer], cp.v_out[layer], out, budgets=cp.budgets)
+    cp.check()
+    want_out = O.decode_attention(P.np64(q_new), P.np64(cp.k_out[layer, :, :S]), P.np64(cp.v_out[layer, :, :S]))
+    np.testing.assert_allclose(P.np64(out), want_out, rtol=1e-4, atol=1e-4)
+    cp.close()

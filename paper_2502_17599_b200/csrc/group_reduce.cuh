@@ -20,7 +20,7 @@ constexpr int kSortWarps = 8;
 constexpr int kSortWarpItems = 256;                          // elements ranked by one warp
 constexpr int kSortBlockItems = kSortWarps * kSortWarpItems; // elements of one block = one column of the digit table
 constexpr int kSegChunk = 128;        // sorted rows walked by one warp
-constexpr int kSegWarps = 8;
+constexpr int kSegWarps = 2;         // small blocks: more of them fit, also beside a resident tensor-core block
 
 // ---- stable radix pass: histogram, scan, scatter ----------------------------------------------
 // table[g][bin][block] <- number of keys of block `block` whose digit is `bin`.
@@ -211,7 +211,7 @@ __device__ __forceinline__ void store_row(T* p, int lane, const float (&x)[E], f
 // grid = (chunks / kSegWarps, heads, 2): blockIdx.z picks the tensor (0 keys, 1 values), so that twice
 // as many warps keep rows in flight; the z = 0 warps also record segment bounds and counts.
 template <typename T, int D>
-__global__ void __launch_bounds__(kSegWarps * 32, 3)
+__global__ void __launch_bounds__(kSegWarps * 32, 9)
 seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ keys,
                   const int32_t* __restrict__ rows, const int32_t* __restrict__ idx_conserved,
                   const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,

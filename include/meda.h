@@ -119,6 +119,24 @@ meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, 
 meda_status meda_window_scores_from_stats(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k,
                                           const float* row_stats, float* scores, float* entropy, void* stream);
 
+/* Eq. 8 as printed, with EVERY prompt row as a query instead of an observation window: the accumulated
+ * score of key j is the column sum of the whole causal attention matrix of prompt encoding,
+ *   scores[g][j] = sum over the query heads h of KV head g and over the rows i >= j of
+ *                  softmax_j(q_i . k / sqrt(head_dim))[h][i][j]      (each KV head's scores sum to group_size * n_tokens).
+ * q_all: device, `dtype`, [n_q_heads][n_tokens][head_dim], the query rows of all prompt tokens (row i sits at
+ * position i and sees keys j <= i); k: device, `dtype`, [n_kv_heads][n_tokens][head_dim].
+ * scores: device fp32 [n_kv_heads][n_tokens], fully overwritten; it can be passed to meda_select_topk /
+ * meda_compress_layer in place of the window's scores.  The cost is that of the prompt's attention itself
+ * (n_tokens^2 / 2 logits per query head, twice: normalisers, then column sums), independent of `window`.
+ * scratch: device memory of at least meda_prompt_scores_scratch_bytes(ctx) bytes, 16-byte aligned, owned by
+ * the caller and free again when the call's work on `stream` has finished (the per-row normalisers live
+ * there; 20 bytes per query head and token, rounded up).  When that size is 0 (fp32 or head_dim != 128: the
+ * rows then go block by block through the context's own scratch) it may be NULL.  A scratch that is too small
+ * returns MEDA_ERR_WORKSPACE and launches nothing. */
+int64_t meda_prompt_scores_scratch_bytes(const meda_ctx* ctx);
+meda_status meda_prompt_scores(meda_ctx* ctx, const void* q_all, const void* k, float* scores, void* scratch,
+                               int64_t scratch_bytes, void* stream);
+
 /* Cross-modal attention entropy of one layer (Eq. 4-6): E_CM = -(E_TV + E_VT), written to entropy[layer].
  *  - The E_TV term uses the text window q_win and its row_stats (from meda_window_scores): one sweep over
  *    the key cache, the same arithmetic as meda_window_scores' own entropy.  For callers that already hold

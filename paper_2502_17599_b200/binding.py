@@ -66,6 +66,8 @@ EXPORTS = {
     "meda_launch_count": (ctypes.c_int64, [ctypes.c_void_p]),
     "meda_window_scores": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
     "meda_window_scores_from_stats": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
+    "meda_prompt_scores_scratch_bytes": (ctypes.c_int64, [ctypes.c_void_p]),
+    "meda_prompt_scores": (ctypes.c_int, [ctypes.c_void_p] * 5 + [ctypes.c_int64, ctypes.c_void_p]),
     "meda_layer_entropy": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 5 +
                            [ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]),
     "meda_decode_attention": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
@@ -209,6 +211,16 @@ class Context:
         _check(self._lib.meda_window_scores_from_stats(self._h, layer, _ptr(q_win), _ptr(k), _ptr(row_stats),
                                                        _ptr(scores), _ptr(entropy), _stream(stream)),
                "meda_window_scores_from_stats")
+
+    def prompt_scores_scratch_bytes(self) -> int:
+        return int(self._lib.meda_prompt_scores_scratch_bytes(self._h))
+
+    def prompt_scores(self, q_all, k, scores, scratch=None, stream=None):
+        """Eq. 8 over every prompt row.  `scratch`: a uint8 device tensor of at least
+        prompt_scores_scratch_bytes() bytes (None only when that is 0)."""
+        nbytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
+        _check(self._lib.meda_prompt_scores(self._h, _ptr(q_all), _ptr(k), _ptr(scores), _ptr(scratch), nbytes,
+                                            _stream(stream)), "meda_prompt_scores")
 
     def layer_entropy(self, layer, q_win, k, row_stats, entropy, q_vis=None, q_vis_pos=None, n_vis_rows=0, stream=None):
         _check(self._lib.meda_layer_entropy(self._h, layer, _ptr(q_win), _ptr(k), _ptr(row_stats), _ptr(q_vis),

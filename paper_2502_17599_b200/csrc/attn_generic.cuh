@@ -26,6 +26,18 @@ __host__ __device__ inline AttnGenericSmem attn_generic_smem(int w, int d, bool 
   return L;
 }
 
+// Where the operands of a launch live when they are not the dense [heads][w] window and [heads][n] cache:
+// a block of query rows inside a longer query tensor, a prefix of the key cache, scores added to what the
+// array holds.  A zero stride means "dense" (w or n rows per head).
+struct AttnView {
+  int rows_from_pos0 = 0;        // 1: query row i sits at position pos0 + i (default: the last w tokens)
+  int pos0 = 0;
+  int64_t q_head_stride = 0;     // rows between consecutive heads of the query tensor
+  int64_t k_head_stride = 0;     // rows between consecutive KV heads of the key cache
+  int64_t score_stride = 0;      // floats between consecutive KV heads of the score array
+  int accumulate = 0;            // 1: scores are added to the array's contents
+};
+
 // Stage one query head [w][d] and one key tile [tile][d] as fp32; rows past n are zero.
 template <typename T>
 __device__ __forceinline__ void stage_q(float* qs, const T* q_h, int w, int d) {
@@ -43,7 +55,9 @@ __device__ __forceinline__ void stage_k(float* ks, const T* k_g, int j0, int n, 
 // s[i][jl] = scale * q_i . k_jl for the staged tile; -inf where the key is past the end of the
 // sequence or hidden from row i by the causal mask.
 __device__ __forceinline__ void tile_logits(float* s, const float* qs, const float* ks, int w, int d,
-                                            int j0, int n, float scale, const int32_t* __restrict__ q_pos = nullptr) {
+                                            int j0, int n, float scale, const int32_t* __restrict__ q_pos = nullptr,
+                                            int pos0 = -1) {
+  if (pos0 < 0) pos0 = n - w;                             // default rows: the last w tokens
   const int jl = threadIdx.x % kGenericKeyTile;
   const int ig = threadIdx.x / kGenericKeyTile;           // 0..3
   constexpr int kRowStep = kAttnThreads / kGenericKeyTile;
@@ -54,7 +68,7 @@ __device__ __forceinline__ void tile_logits(float* s, const float* qs, const flo
     float acc = 0.f;
 #pragma unroll 8
     for (int t = 0; t < d; ++t) acc = fmaf(qr[t], kr[t], acc);
-    bool visible = (j < n) && (j <= (q_pos ? q_pos[i] : n - w + i));      // default rows: the last w tokens
+    bool visible = (j < n) && (j <= (q_pos ? q_pos[i] : pos0 + i));
     s[i * kGenericKeyTile + jl] = visible ? acc * scale : -INFINITY;
   }
 }
@@ -67,7 +81,8 @@ template <typename T>
 __global__ void __launch_bounds__(kAttnThreads)
 stats_partial_kernel(const T* __restrict__ q_win, const T* __restrict__ k, const uint8_t* __restrict__ modality,
                      float* __restrict__ partial, int hq, int group, int n, int w, int d, float scale,
-                     const int32_t* __restrict__ q_pos = nullptr, int subset = MEDA_VISUAL, int subset_only = 0) {
+                     const int32_t* __restrict__ q_pos = nullptr, int subset = MEDA_VISUAL, int subset_only = 0,
+                     AttnView view = AttnView()) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const AttnGenericSmem L = attn_generic_smem(w, d, false);
   float* qs = reinterpret_cast<float*>(smem_raw + L.q_off);
@@ -78,9 +93,10 @@ stats_partial_kernel(const T* __restrict__ q_win, const T* __restrict__ k, const
   const int chunks = gridDim.x;
   const int n_tiles = (n + kGenericKeyTile - 1) / kGenericKeyTile;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const T* k_g = k + (size_t)g * n * d;
+  const T* k_g = k + (size_t)g * (view.k_head_stride ? view.k_head_stride : n) * d;
+  const int pos0 = view.rows_from_pos0 ? view.pos0 : -1;
 
-  stage_q<T>(qs, q_win + (size_t)h * w * d, w, d);
+  stage_q<T>(qs, q_win + (size_t)h * (view.q_head_stride ? view.q_head_stride : w) * d, w, d);
   // running (m, z) of every window row, updated by lane 0 of the warp that owns the row
   __shared__ float rs[kMaxWindow][4];
   for (int i = threadIdx.x; i < w; i += blockDim.x) {
@@ -98,7 +114,7 @@ stats_partial_kernel(const T* __restrict__ q_win, const T* __restrict__ k, const
     }
     stage_k<T>(ks, k_g, j0, n, d);
     __syncthreads();
-    tile_logits(s, qs, ks, w, d, j0, n, scale, q_pos);
+    tile_logits(s, qs, ks, w, d, j0, n, scale, q_pos, pos0);
     __syncthreads();
     for (int i = warp; i < w; i += kAttnThreads / 32) {
       float a0 = s[i * kGenericKeyTile + lane], a1 = s[i * kGenericKeyTile + lane + 32];
@@ -166,7 +182,8 @@ scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, cons
                       const float* __restrict__ row_stats, float* __restrict__ scores,
                       float* __restrict__ ent_partial, int hq, int group, int n, int w, int d, float scale,
                       int entropy_mode, int want_scores, int want_entropy,
-                      const int32_t* __restrict__ q_pos = nullptr, int subset = MEDA_VISUAL) {
+                      const int32_t* __restrict__ q_pos = nullptr, int subset = MEDA_VISUAL,
+                      AttnView view = AttnView()) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const AttnGenericSmem L = attn_generic_smem(w, d, true);
   float* qs = reinterpret_cast<float*>(smem_raw + L.q_off);
@@ -184,6 +201,10 @@ scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, cons
   const bool in_range = j < n;
   const bool visual = in_range && modality[in_range ? j : 0] == subset;      // "in the subset the entropy is taken over"
   const float inv_hq = 1.f / (float)hq;
+  const int pos0 = view.rows_from_pos0 ? view.pos0 : -1;
+  const size_t q_stride = (size_t)(view.q_head_stride ? view.q_head_stride : w) * d;
+  const size_t k_stride = (size_t)(view.k_head_stride ? view.k_head_stride : n) * d;
+  const size_t score_stride = view.score_stride ? (size_t)view.score_stride : (size_t)n;
   if (!want_scores && !__syncthreads_or(visual ? 1 : 0)) {
     // entropy only, and no key of this tile is in the subset: nothing to add
     if (threadIdx.x == 0) ent_partial[blockIdx.x] = 0.f;
@@ -197,10 +218,10 @@ scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, cons
   for (int h = 0; h < hq; ++h) {
     const int g = h / group;
     __syncthreads();
-    stage_q<T>(qs, q_win + (size_t)h * w * d, w, d);
-    if (h % group == 0) stage_k<T>(ks, k + (size_t)g * n * d, j0, n, d);
+    stage_q<T>(qs, q_win + (size_t)h * q_stride, w, d);
+    if (h % group == 0) stage_k<T>(ks, k + (size_t)g * k_stride, j0, n, d);
     __syncthreads();
-    tile_logits(s, qs, ks, w, d, j0, n, scale, q_pos);
+    tile_logits(s, qs, ks, w, d, j0, n, scale, q_pos, pos0);
     // each thread revisits only the logits it wrote itself: no barrier needed here
     float part = 0.f;
     for (int i = ig; i < w; i += kRowStep) {
@@ -222,7 +243,10 @@ scores_entropy_kernel(const T* __restrict__ q_win, const T* __restrict__ k, cons
         group_score += colsum[jl] + colsum[kGenericKeyTile + jl] + colsum[2 * kGenericKeyTile + jl] +
                        colsum[3 * kGenericKeyTile + jl];
         if (h % group == group - 1) {
-          if (in_range) scores[(size_t)g * n + j] = group_score;
+          if (in_range) {
+            float* out = scores + (size_t)g * score_stride + j;
+            *out = view.accumulate ? *out + group_score : group_score;
+          }
           group_score = 0.f;
         }
       }

@@ -17,6 +17,7 @@
 #include "group_reduce.cuh"
 #include "merge_generic.cuh"
 #include "nearest_sm100.cuh"
+#include "prompt_scores_sm100.cuh"
 #include "select.cuh"
 
 using namespace meda;
@@ -322,6 +323,101 @@ meda_status launch_evt(meda_ctx* ctx, int32_t layer, const void* q_vis, const in
   {
     LaunchScope scope(ctx, MEDA_K_ENTROPY_FINAL, st);
     entropy_finalize_kernel<<<1, 256, 0, st>>>(ctx->ws.ent_partial, tiles, ctx->ws.row_stats_vis, rows, entropy + layer, 1);
+  }
+  return launch_status();
+}
+
+// ---- Eq. 8 over every prompt row ---------------------------------------------------------------
+// Rows per head of the per-row reference array: a multiple of 128 so that a streamed tile of query
+// rows never reads past it.
+int64_t prompt_n_pad(const meda_ctx* ctx) { return ((int64_t)ctx->cfg.n_tokens + 127) / 128 * 128; }
+
+int64_t prompt_scratch_bytes(const meda_ctx* ctx) {
+  if (!ctx->fast) return 0;                            // the CUDA-core path works inside the context's own scratch
+  return (int64_t)ctx->cfg.n_q_heads * prompt_n_pad(ctx) * (sizeof(float) + 2 * sizeof(float2));
+}
+
+// bf16, head_dim 128: two launches of the streaming tensor-core pipeline over the causal half of the matrix.
+meda_status launch_prompt_fast(meda_ctx* ctx, const void* q_all, const void* k, float* scores, void* scratch,
+                               cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  if (((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(q_all) | reinterpret_cast<uintptr_t>(scratch)) & 15u) != 0)
+    return MEDA_ERR_INVALID_ARG;
+  CUtensorMap map_q, map_k;
+  if (!make_rows_map(ctx, &map_q, q_all, c.n_tokens, c.n_q_heads, c.n_tokens, 128) ||
+      !make_rows_map(ctx, &map_k, k, c.n_tokens, c.n_kv_heads, c.n_tokens, 128))
+    return MEDA_ERR_CUDA;
+  const int n_pad = (int)prompt_n_pad(ctx);
+  float* ref = static_cast<float*>(scratch);
+  float2* partial = reinterpret_cast<float2*>(ref + (size_t)c.n_q_heads * n_pad);
+  const float sc2 = kLog2e / sqrtf((float)c.head_dim);
+  const int blocks256 = (c.n_tokens + 255) / 256;
+  {
+    PromptStatsPolicy::Params prm;
+    prm.partial = partial;
+    prm.n = c.n_tokens; prm.n_pad = n_pad; prm.hq = c.n_q_heads; prm.group = ctx->group;
+    prm.row_blocks = blocks256;
+    prm.sc2 = sc2;
+    LaunchScope scope(ctx, MEDA_K_STATS, st);
+    umma_stream_kernel<PromptStatsPolicy><<<(int)std::min<int64_t>((int64_t)blocks256 * c.n_q_heads, ctx->sm_count),
+                                            us_threads<PromptStatsPolicy>(), StreamShared<PromptStatsPolicy>::alloc, st>>>(
+        map_q, map_k, prm, ctx->ws.status);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
+    prompt_ref_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(partial, ref, c.n_q_heads, c.n_tokens, n_pad);
+  }
+  {
+    PromptSweepPolicy::Params prm;
+    prm.ref = ref;
+    prm.scores = scores;
+    prm.n = c.n_tokens; prm.n_pad = n_pad; prm.hq = c.n_q_heads; prm.group = ctx->group;
+    prm.n_blocks = blocks256;
+    prm.sc2 = sc2;
+    LaunchScope scope(ctx, MEDA_K_SWEEP, st);
+    umma_stream_kernel<PromptSweepPolicy><<<std::min(blocks256, ctx->sm_count), us_threads<PromptSweepPolicy>(),
+                                            StreamShared<PromptSweepPolicy>::alloc, st>>>(map_k, map_q, prm, ctx->ws.status);
+  }
+  return launch_status();
+}
+
+// Any dtype and head dimension: the prompt rows in blocks of `window` rows through the CUDA-core kernels
+// of the observation window; block b sees the keys up to its last row and adds its column sums.
+template <typename T>
+meda_status launch_prompt_generic(meda_ctx* ctx, const void* q_all, const void* k, float* scores, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  const float scale = 1.0f / sqrtf((float)c.head_dim);
+  MEDA_CUDA_TRY(cudaMemsetAsync(scores, 0, sizeof(float) * (size_t)c.n_kv_heads * c.n_tokens, st));
+  for (int p0 = 0; p0 < c.n_tokens; p0 += c.window) {
+    const int rows = std::min(c.window, c.n_tokens - p0);
+    const int n_seen = p0 + rows;
+    const int tiles = generic_tiles(n_seen);
+    const int chunks = std::min(kStatsChunks, tiles);
+    AttnView view;
+    view.rows_from_pos0 = 1;
+    view.pos0 = p0;
+    view.q_head_stride = c.n_tokens;
+    view.k_head_stride = c.n_tokens;
+    view.score_stride = c.n_tokens;
+    view.accumulate = 1;
+    const T* q_block = static_cast<const T*>(q_all) + (size_t)p0 * c.head_dim;
+    {
+      LaunchScope scope(ctx, MEDA_K_STATS, st);
+      stats_partial_kernel<T><<<dim3(chunks, c.n_q_heads), kAttnThreads, attn_generic_smem(rows, c.head_dim, false).total, st>>>(
+          q_block, static_cast<const T*>(k), ctx->ws.modality, ctx->ws.stats_partial, c.n_q_heads, ctx->group, n_seen,
+          rows, c.head_dim, scale, nullptr, MEDA_VISUAL, 0, view);
+    }
+    {
+      LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
+      stats_combine_kernel<<<(c.n_q_heads * rows + 7) / 8, 256, 0, st>>>(ctx->ws.stats_partial, ctx->ws.row_stats_vis,
+                                                                         chunks, c.n_q_heads * rows);
+    }
+    {
+      LaunchScope scope(ctx, MEDA_K_SWEEP, st);
+      scores_entropy_kernel<T><<<tiles, kAttnThreads, attn_generic_smem(rows, c.head_dim, true).total, st>>>(
+          q_block, static_cast<const T*>(k), ctx->ws.modality, ctx->ws.row_stats_vis, scores, ctx->ws.ent_partial,
+          c.n_q_heads, ctx->group, n_seen, rows, c.head_dim, scale, c.entropy_mode, 1, 0, nullptr, MEDA_VISUAL, view);
+    }
   }
   return launch_status();
 }
@@ -695,6 +791,12 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     if (st == MEDA_OK && cudaFuncSetAttribute(nearest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)NearestSmem::alloc) != cudaSuccess)
       st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<PromptStatsPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)StreamShared<PromptStatsPolicy>::alloc) != cudaSuccess)
+      st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<PromptSweepPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)StreamShared<PromptSweepPolicy>::alloc) != cudaSuccess)
+      st = MEDA_ERR_CUDA;
   }
   if (st == MEDA_OK) st = carve(&ws.target, hkv * n, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.idx_less, hkv * n, &ws.bytes);
@@ -812,6 +914,19 @@ meda_status meda_window_scores_from_stats(meda_ctx* ctx, int32_t layer, const vo
   if (ctx->fast_attn) return launch_sweep_fast(ctx, layer, q_win, k, row_stats, scores, entropy, st);
   if (ctx->cfg.dtype == MEDA_F32) return launch_sweep<float>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
   return launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+}
+
+int64_t meda_prompt_scores_scratch_bytes(const meda_ctx* ctx) { return ctx ? prompt_scratch_bytes(ctx) : 0; }
+
+meda_status meda_prompt_scores(meda_ctx* ctx, const void* q_all, const void* k, float* scores, void* scratch,
+                               int64_t scratch_bytes, void* stream) {
+  if (!ctx || !q_all || !k || !scores) return MEDA_ERR_INVALID_ARG;
+  const int64_t need = prompt_scratch_bytes(ctx);
+  if (need > 0 && (!scratch || scratch_bytes < need)) return MEDA_ERR_WORKSPACE;
+  cudaStream_t st = as_stream(stream);
+  if (ctx->fast) return launch_prompt_fast(ctx, q_all, k, scores, scratch, st);
+  return ctx->cfg.dtype == MEDA_F32 ? launch_prompt_generic<float>(ctx, q_all, k, scores, st)
+                                    : launch_prompt_generic<__nv_bfloat16>(ctx, q_all, k, scores, st);
 }
 
 meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,

@@ -229,10 +229,28 @@ def make_layer(wl: Workload, layer: int, device="cpu"):
     """
     k = _cache_tensor(wl, layer, 0, device, scale_salient=True)
     v = _cache_tensor(wl, layer, 1, device, scale_salient=False)
+    return make_layer_queries(wl, layer, device), k, v
+
+
+def make_layer_queries(wl: Workload, layer: int, device="cpu"):
+    """q_win [Hq, w, d] of make_layer alone."""
     hq, w, d = wl.n_q_heads, wl.window, wl.head_dim
     tau = layer_temperature(wl, layer)
-    q = (tau * normal(stream_key(wl.seed, layer, 2), 0, hq * w * d, device)).view(hq, w, d).to(wl.torch_dtype)
-    return q, k, v
+    return (tau * normal(stream_key(wl.seed, layer, 2), 0, hq * w * d, device)).view(hq, w, d).to(wl.torch_dtype)
+
+
+def make_prompt_queries(wl: Workload, layer: int, device="cpu"):
+    """q_all [Hq, n, d] in the workload's dtype: a query row for every prompt token (Eq. 8 without the
+    observation-window restriction).  Same distribution as the window's queries; the last `window` rows
+    are the rows make_layer returns."""
+    hq, n, w, d = wl.n_q_heads, wl.n_tokens, wl.window, wl.head_dim
+    tau = layer_temperature(wl, layer)
+    q = torch.empty((hq, n, d), dtype=wl.torch_dtype, device=device)
+    key = stream_key(wl.seed, layer, 4)
+    for h in range(hq):
+        q[h] = (tau * normal(key, h * n * d, n * d, device)).view(n, d).to(wl.torch_dtype)
+    q[:, n - w:] = make_layer_queries(wl, layer, device)
+    return q
 
 
 def make_visual_queries(wl: Workload, layer: int, n_rows: int, device="cpu"):

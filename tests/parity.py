@@ -143,3 +143,15 @@ def compare_merged(got_k, got_v, got_counts, k_g, v_g, conserved, less, target, 
             assert (err <= MERGE_F32_RTOL * np.abs(want) + 1e-6).all(), float(err.max())
             stats["max_abs"] = max(stats["max_abs"], float(err.max()) if err.size else 0.0)
     return stats
+
+
+def oracle_prompt_scores(q_all: np.ndarray, k: np.ndarray, block: int = 1024) -> np.ndarray:
+    """Eq. 8 over every prompt row with the oracle: its window_scores evaluated on consecutive blocks of
+    query rows at their own positions and added up (the score is a sum over rows), so that the n x n
+    matrix never has to exist at once.  q_all [Hq, n, d], k [Hkv, n, d] -> [Hkv, n]."""
+    n = k.shape[1]
+    out = np.zeros((k.shape[0], n))
+    for p0 in range(0, n, block):
+        pos = np.arange(p0, min(p0 + block, n))
+        out[:, : pos[-1] + 1] += O.window_scores(q_all[:, pos], k[:, : pos[-1] + 1], q_pos=pos)
+    return out

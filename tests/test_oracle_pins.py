@@ -452,3 +452,19 @@ def test_decode_attention_closed_forms_and_bruteforce():
             want[h][t] = sum(w[j] * v[g][j][t] for j in range(s_rows)) / z
     np.testing.assert_allclose(O.decode_attention(q, k, v), want, atol=1e-12)
 
+
+
+def test_blockwise_prompt_scores_helper_and_prompt_query_generator():
+    """The row-block evaluation the full-size GPU test uses equals the oracle's one-shot result with the
+    window equal to the prompt, and the prompt-wide query generator ends in the observation window's rows."""
+    import parity as P
+    from paper_2502_17599_b200 import workloads as W
+    q = RNG.normal(size=(4, 37, 5))
+    k = RNG.normal(size=(2, 37, 5))
+    np.testing.assert_allclose(P.oracle_prompt_scores(q, k, block=8), O.window_scores(q, k), rtol=1e-12)
+    wl = W.small_variant()
+    q_all = W.make_prompt_queries(wl, 1)
+    q_win, _, _ = W.make_layer(wl, 1)
+    assert q_all.shape == (wl.n_q_heads, wl.n_tokens, wl.head_dim) and q_all.dtype == q_win.dtype
+    assert torch.equal(q_all[:, -wl.window:], q_win)
+    assert not torch.equal(q_all[0, :wl.window], q_all[1, :wl.window])

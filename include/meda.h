@@ -129,8 +129,8 @@ meda_status meda_window_scores_from_stats(meda_ctx* ctx, int32_t layer, const vo
  * meda_compress_layer in place of the window's scores.  The cost is that of the prompt's attention itself
  * (n_tokens^2 / 2 logits per query head, twice: normalisers, then column sums), independent of `window`.
  * scratch: device memory of at least meda_prompt_scores_scratch_bytes(ctx) bytes, 16-byte aligned, owned by
- * the caller and free again when the call's work on `stream` has finished (the per-row normalisers live
- * there; 20 bytes per query head and token, rounded up).  When that size is 0 (fp32 or head_dim != 128: the
+ * the caller and free again when the call's work on `stream` has finished (the per-row normalisers and the
+ * partial scores live there: 20 bytes per query head and token or a little more).  When that size is 0 (fp32 or head_dim != 128: the
  * rows then go block by block through the context's own scratch) it may be NULL.  A scratch that is too small
  * returns MEDA_ERR_WORKSPACE and launches nothing. */
 int64_t meda_prompt_scores_scratch_bytes(const meda_ctx* ctx);

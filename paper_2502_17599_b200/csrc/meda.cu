@@ -332,9 +332,20 @@ meda_status launch_evt(meda_ctx* ctx, int32_t layer, const void* q_vis, const in
 // rows never reads past it.
 int64_t prompt_n_pad(const meda_ctx* ctx) { return ((int64_t)ctx->cfg.n_tokens + 127) / 128 * 128; }
 
+// Row runs per key block of the column-sum pass: enough (key block, KV head, run) units for about six per SM.
+int prompt_splits(const meda_ctx* ctx) {
+  const int64_t units = (int64_t)((ctx->cfg.n_tokens + 255) / 256) * ctx->cfg.n_kv_heads;
+  return (int)std::max<int64_t>(1, std::min<int64_t>(8, (6 * (int64_t)ctx->sm_count + units - 1) / units));
+}
+
+// Per-row references, then one region that first holds the two partial normalisers of every row and later
+// the partial scores of every key.
 int64_t prompt_scratch_bytes(const meda_ctx* ctx) {
   if (!ctx->fast) return 0;                            // the CUDA-core path works inside the context's own scratch
-  return (int64_t)ctx->cfg.n_q_heads * prompt_n_pad(ctx) * (sizeof(float) + 2 * sizeof(float2));
+  const int64_t n_pad = prompt_n_pad(ctx);
+  const int64_t stats_part = 2 * (int64_t)sizeof(float2) * ctx->cfg.n_q_heads * n_pad;
+  const int64_t score_part = 2 * (int64_t)sizeof(float) * prompt_splits(ctx) * ctx->cfg.n_kv_heads * n_pad;
+  return (int64_t)sizeof(float) * ctx->cfg.n_q_heads * n_pad + std::max(stats_part, score_part);
 }
 
 // bf16, head_dim 128: two launches of the streaming tensor-core pipeline over the causal half of the matrix.
@@ -367,16 +378,29 @@ meda_status launch_prompt_fast(meda_ctx* ctx, const void* q_all, const void* k, 
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
     prompt_ref_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(partial, ref, c.n_q_heads, c.n_tokens, n_pad);
   }
+  const int splits = prompt_splits(ctx);
+  float* score_part = reinterpret_cast<float*>(partial);     // the partial normalisers are spent once ref is written
   {
     PromptSweepPolicy::Params prm;
     prm.ref = ref;
-    prm.scores = scores;
-    prm.n = c.n_tokens; prm.n_pad = n_pad; prm.hq = c.n_q_heads; prm.group = ctx->group;
+    prm.partial = score_part;
+    prm.n = c.n_tokens; prm.n_pad = n_pad; prm.hq = c.n_q_heads; prm.hkv = c.n_kv_heads; prm.group = ctx->group;
     prm.n_blocks = blocks256;
+    prm.splits = splits;
+    prm.full_blocks = 0;
+    int64_t units = 0;
+    for (int blk = 0; blk < blocks256; ++blk) {
+      if (prompt_block_tiles(c.n_tokens, blk) >= splits) prm.full_blocks = blk + 1;
+      units += (int64_t)c.n_kv_heads * prompt_block_splits(c.n_tokens, blk, splits);
+    }
     prm.sc2 = sc2;
     LaunchScope scope(ctx, MEDA_K_SWEEP, st);
-    umma_stream_kernel<PromptSweepPolicy><<<std::min(blocks256, ctx->sm_count), us_threads<PromptSweepPolicy>(),
+    umma_stream_kernel<PromptSweepPolicy><<<(int)std::min<int64_t>(units, ctx->sm_count), us_threads<PromptSweepPolicy>(),
                                             StreamShared<PromptSweepPolicy>::alloc, st>>>(map_k, map_q, prm, ctx->ws.status);
+  }
+  {
+    LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
+    prompt_sum_kernel<<<2 * ctx->sm_count, 256, 0, st>>>(score_part, scores, c.n_kv_heads, c.n_tokens, splits);
   }
   return launch_status();
 }

@@ -12,7 +12,9 @@
 //                     sums exp2(t - ref[row]) over the rows that see it.  With ref = max + log2(sum)
 //                     that exponential already is the softmax probability: one fused multiply-add,
 //                     one exp2 and one add per logit.  The query heads of a KV head follow each other
-//                     in the same block, so a key's score is complete inside one thread.
+//                     in the same block; the rows a key block streams are cut into a few runs, and two
+//                     epilogue groups take alternate row tiles: prompt_sum_kernel adds those partial
+//                     scores in a fixed order.
 //
 // Logits are kept in base-2 units: t = (q.k) * scale * log2(e).
 #pragma once
@@ -151,46 +153,74 @@ prompt_ref_kernel(const float2* __restrict__ partial, float* __restrict__ ref, i
 // ---------------------------------------------------------------------------------------------
 // Pass 2: column sums
 // ---------------------------------------------------------------------------------------------
+// The rows a 256-key block streams (from its first key to the end of the prompt) are cut into up to
+// `splits` contiguous runs of row tiles, so that short prompts still fill the GPU; a block with fewer
+// row tiles than that has one run per tile.
+__host__ __device__ inline int prompt_block_tiles(int n, int blk) { return (n - blk * 256 + 127) / 128; }
+__host__ __device__ inline int prompt_block_splits(int n, int blk, int splits) {
+  const int t = prompt_block_tiles(n, blk);
+  return t < splits ? t : splits;
+}
+
 struct PromptSweepPolicy {
   struct Params {
     const float* ref;            // [Hq][n_pad]
-    float* scores;               // [Hkv][n]
-    int n, n_pad, hq, group;
+    float* partial;              // [splits * 2][Hkv][n]: one slot per (row run, epilogue group)
+    int n, n_pad, hq, hkv, group;
     int n_blocks;                // ceil(n / 256)
+    int splits;                  // row runs per key block (1..8)
+    int full_blocks;             // key blocks with at least `splits` row tiles: blocks 0 .. full_blocks - 1
     float sc2;
   };
   static constexpr int kABuffers = 2;
   static constexpr int kBStages = 3;
-  static constexpr int kEpilogueGroups = 1;
+  static constexpr int kEpilogueGroups = 2;
   static constexpr uint32_t kExtraBytes = 0;
   static constexpr uint32_t kItemExtraBytes = 0;
 
   __device__ static bool active(const Params&) { return true; }
-  // A block takes whole 256-key blocks (the first ones have the most rows to stream) and walks all
-  // query heads of a key block back to back.
+  // A unit = (key block, KV head, row run), longest first (block 0 streams the most rows); the thread
+  // block that takes a unit walks the query heads of its KV head back to back, one item each.
   __device__ static bool get_item(const Params& p, int it, StreamItem& o) {
-    const int blk = blockIdx.x + (it / p.hq) * gridDim.x;
-    if (blk >= p.n_blocks) return false;
-    const int h = it % p.hq;
+    int u = blockIdx.x + (it / p.group) * gridDim.x;
+    const int per_full = p.hkv * p.splits;
+    int blk, runs;
+    if (u < p.full_blocks * per_full) {
+      blk = u / per_full;
+      u -= blk * per_full;
+      runs = p.splits;
+    } else {
+      u -= p.full_blocks * per_full;
+      for (blk = p.full_blocks; blk < p.n_blocks; ++blk) {      // at most splits / 2 short blocks at the end
+        runs = prompt_block_splits(p.n, blk, p.splits);
+        if (u < p.hkv * runs) break;
+        u -= p.hkv * runs;
+      }
+      if (blk >= p.n_blocks) return false;
+    }
+    const int g = u / runs, run = u % runs;
+    const int tiles = prompt_block_tiles(p.n, blk);
+    const int t_lo = run * tiles / runs, t_hi = (run + 1) * tiles / runs;     // runs <= tiles: never empty
     o.a_row = blk * 256;
-    o.a_head = h / p.group;
-    o.b_row = blk * 256;                             // earlier rows see none of these keys
-    o.b_head = h;
-    o.n_tiles = (p.n - o.b_row + 127) / 128;         // rows past n read as zeros and carry the "no row" reference
+    o.a_head = g;
+    o.b_row = blk * 256 + t_lo * 128;                // earlier rows see none of these keys
+    o.b_head = g * p.group + it % p.group;
+    o.n_tiles = t_hi - t_lo;                         // rows past n read as zeros and carry the "no row" reference
     o.last_n = 128;
     o.m_tiles = (p.n - o.a_row > 128) ? 2 : 1;
-    o.u0 = h;
-    o.u1 = blk;
+    o.u0 = o.b_head;
+    o.u1 = run;
     return true;
   }
 
   struct Epilogue {
-    int lane, row_in_block;
-    float score;                 // this thread's key, summed over the tiles and heads of its KV head so far
+    int lane, row_in_block, egroup;
+    float score;                 // this thread's key, summed over the tiles and heads of the unit so far
     float s0, s1, s2, s3;        // partial sums inside one tile: small addends meet a small running sum
     __device__ void init(const Params&, unsigned char*, int ewarp, int lane_) {
       lane = lane_;
-      row_in_block = (ewarp / 4) * 128 + ((ewarp + 2) % 4) * 32 + lane_;
+      egroup = ewarp / kUsEpilogueWarps;
+      row_in_block = ((ewarp % kUsEpilogueWarps) / 4) * 128 + ((ewarp + 2) % 4) * 32 + lane_;
       score = 0.f;
     }
     __device__ void item_begin(const Params&, const StreamItem&, const unsigned char*) {}
@@ -216,35 +246,40 @@ struct PromptSweepPolicy {
       const int warp_first = j - lane;                  // the warp's first key is seen by the most rows
       const int r_tile = it.b_row + tile * 128;
       const float4* ref4 = reinterpret_cast<const float4*>(p.ref + (size_t)it.u0 * p.n_pad + r_tile);
-      // two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced
-      uint32_t ra[32], rb[32];
-      int c = 0;
-      while (c < 4 && r_tile + 32 * c + 31 < warp_first) ++c;      // rows that see no key of the warp
-      if (c == 4) return;
       s0 = s1 = s2 = s3 = 0.f;
-      sm100::tmem_ld_32x32_issue(taddr + 32u * c, ra);
+      // one chunk in registers at a time (sixteen epilogue warps hide the load latency for each other, and
+      // a block of this size has no registers for a second buffer)
+      uint32_t acc[32];
 #pragma unroll 1
-      for (; c < 4; c += 2) {
+      for (int c = 0; c < 4; ++c) {
+        if (r_tile + 32 * c + 31 < warp_first) continue;          // rows that see no key of the warp
+        sm100::tmem_ld_32x32_issue(taddr + 32u * c, acc);
         sm100::tmem_ld_wait();
-        sm100::tmem_ld_pin(ra);
-        if (c + 1 < 4) sm100::tmem_ld_32x32_issue(taddr + 32u * (c + 1), rb);
-        if (valid) chunk(p, ra, ref4 + 8 * c, r_tile + 32 * c, j);
-        if (c + 1 < 4) {
-          sm100::tmem_ld_wait();
-          sm100::tmem_ld_pin(rb);
-          if (c + 2 < 4) sm100::tmem_ld_32x32_issue(taddr + 32u * (c + 2), ra);
-          if (valid) chunk(p, rb, ref4 + 8 * (c + 1), r_tile + 32 * (c + 1), j);
-        }
+        sm100::tmem_ld_pin(acc);
+        if (valid) chunk(p, acc, ref4 + 8 * c, r_tile + 32 * c, j);
       }
       score += (s0 + s1) + (s2 + s3);
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {
       if (it.u0 % p.group != p.group - 1) return;       // more heads of this KV head follow
       const int j = it.a_row + row_in_block;
-      if (j < p.n) p.scores[(size_t)(it.u0 / p.group) * p.n + j] = score;
+      if (j < p.n) p.partial[((size_t)(it.u1 * 2 + egroup) * p.hkv + it.u0 / p.group) * p.n + j] = score;
       score = 0.f;
     }
   };
 };
+
+// scores[g][j] = the slots of key j's block added in slot order (row run by row run, epilogue group 0 then 1).
+__global__ void __launch_bounds__(256)
+prompt_sum_kernel(const float* __restrict__ partial, float* __restrict__ scores, int hkv, int n, int splits) {
+  const size_t total = (size_t)hkv * n;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    const int j = (int)(e % n);
+    const int slots = 2 * prompt_block_splits(n, j / 256, splits);
+    float acc = 0.f;
+    for (int s = 0; s < slots; ++s) acc += partial[(size_t)s * total + e];
+    scores[e] = acc;
+  }
+}
 
 }  // namespace meda

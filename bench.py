@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="skip the decoding-step context measurement")
+    ap.add_argument("--no-prompt-scores", action="store_true",
+                    help="skip the context measurement of Eq. 8 taken over every prompt row (one layer)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     return ap.parse_args()
 
@@ -360,6 +362,33 @@ def run_ours(args):
                   "GB/s_compressed": bytes_c / ms_c / 1e6, "GB/s_full": bytes_f / ms_f / 1e6}
         cp.check()
 
+    # context: Eq. 8 as printed (every prompt row a query, no observation window), one layer
+    prompt_ctx = None
+    if not args.no_prompt_scores:
+        q_all = W.make_prompt_queries(wl, 0, "cuda")
+        scratch = torch.empty(max(cp.ctx.prompt_scores_scratch_bytes(), 16), dtype=torch.uint8, device="cuda")
+        sc_all = torch.zeros((wl.n_kv_heads, wl.n_tokens), dtype=torch.float32, device="cuda")
+        cp.ctx.prompt_scores(q_all, ks[0], sc_all, scratch)                  # warm-up
+        cp.check()
+        cp.ctx.profile_read()
+        cp.ctx.profile_enable(True)
+        reps = 2
+        for _ in range(reps):
+            cp.ctx.prompt_scores(q_all, ks[0], sc_all, scratch)
+        cp.check()
+        pr = {k_: v_[0] / reps for k_, v_ in cp.ctx.profile_read().items() if v_[1]}
+        cp.ctx.profile_enable(False)
+        logits = wl.n_q_heads * wl.n_tokens * (wl.n_tokens + 1) / 2
+        ms_layer = sum(pr.values())
+        sfu = 148 * 16 * ((clocks or {}).get("sm_max_mhz") or 1965.0) * 1e6
+        prompt_ctx = {"what": "scores of Eq. 8 with every prompt row as a query (column sums of the causal attention), "
+                              "one layer: normalisers pass, column-sum pass and two small kernels",
+                      "ms_per_layer": ms_layer, "ms_normalisers": pr.get("stats"), "ms_column_sums": pr.get("sweep"),
+                      "logits_per_pass": logits, "TFLOP/s": 2 * 2 * logits * wl.head_dim / (ms_layer * 1e-3) / 1e12,
+                      "exp2/s": 2 * logits / (ms_layer * 1e-3), "frac_of_sfu_peak": 2 * logits / (ms_layer * 1e-3) / sfu,
+                      "window_scores_ms_per_layer": (per_layer_window_ms(prof, L))}
+        del q_all, scratch, sc_all
+
     # end-to-end leg: pinned host inputs -> device -> pass -> compacted caches back to the host
     e2e = None
     if not args.no_e2e:
@@ -449,10 +478,18 @@ def run_ours(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roof, "kernels": per_class, "kernel_rooflines": extra, "cpu_baseline": cpu,
         "budgets_min_max": [int(budgets.min()), int(budgets.max())], "decode_context": decode,
+        "prompt_scores_context": prompt_ctx,
     }
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def per_layer_window_ms(prof, n_layers):
+    """Device time per layer of the observation-window phase A in the profiled steps (for comparison)."""
+    ms = sum(prof[c][0] for c in ("stats", "stats_combine", "sweep", "entropy_final") if c in prof and prof[c][1])
+    cnt = prof["sweep"][1] if "sweep" in prof and prof["sweep"][1] else 0
+    return ms / cnt if cnt else None
 
 
 def main():

@@ -87,6 +87,40 @@ def test_entropy_closed_forms_on_device():
     ctx.close()
 
 
+@pytest.mark.parametrize("window", [24, 32, 64])
+@pytest.mark.parametrize("modality", [0, 1])
+def test_single_modality_prompts_on_both_phase_a_paths(window, modality):
+    """A prompt of text alone has no cross-modal attention (entropy 0); a prompt of visual tokens alone has
+    text-to-vision attention equal to the whole attention.  Windows 32 and 64 take the tensor-core kernels,
+    24 the CUDA-core ones; scores, normalisers and entropy against the oracle, then a selection."""
+    base = W.small_variant(window=window, seed=12)
+    wl = base.with_(name=f"one_modality_{modality}", spans=((0, base.n_tokens, modality),), frame_tokens=0)
+    mod = wl.modality().numpy()
+    ctx = make_ctx(wl)
+    buf = P.GpuBuffers(wl)
+    (q, k, v), (qh, kh, vh) = P.layer_inputs(wl, 0, "cuda")
+    ctx.window_scores(0, q, k, buf.row_stats, buf.scores, buf.entropy)
+    ctx.check()
+    P.assert_row_stats_close(P.np64(buf.row_stats), O.row_stats(qh, kh, mod))
+    a_s = O.window_scores(qh, kh)
+    P.assert_scores_close(P.np64(buf.scores), a_s)
+    want_e = O.cross_modal_entropy(qh, kh, mod)
+    if modality == 0:
+        assert want_e == 0.0 and float(buf.entropy[0]) == 0.0
+    else:
+        assert want_e > 0.0
+        P.assert_entropy_close(float(buf.entropy[0]), want_e)
+    S = wl.n_tokens // 3
+    M = (3 * S) // 4
+    budgets = torch.tensor([[S, M, S - M]] * wl.n_layers, dtype=torch.int32, device="cuda")
+    ctx.select_topk(0, buf.scores, budgets, buf.idx_c, buf.idx_less, buf.cap)
+    ctx.check()
+    got = P.np64(buf.scores)
+    for g in range(wl.n_kv_heads):
+        P.compare_selection(buf.idx_c[g, :S].cpu().numpy(), got[g], mod, M, S - M)
+    ctx.close()
+
+
 @pytest.mark.parametrize("alloc_mode", [0, 1])
 def test_allocate_budgets_bit_exact(alloc_mode):
     rng = np.random.default_rng(7)

@@ -261,7 +261,17 @@ def test_merge_special_cases_on_device():
     ctx.close()
 
 
-@pytest.mark.parametrize("wl", small_cases(), ids=lambda w: w.name)
+def reseeded_cases():
+    """The first three benchmark configurations under two more seeds (two layers each of the larger ones)."""
+    out = []
+    for seed in (1, 2):
+        out.append(W.WORKLOADS["tiny"].with_(name=f"tiny_seed{seed}", seed=seed))
+        out.append(W.WORKLOADS["multi_image_8k"].with_(name=f"multi_image_8k_2l_seed{seed}", n_layers=2, seed=seed))
+        out.append(W.WORKLOADS["long_video_19k"].with_(name=f"long_video_19k_2l_seed{seed}", n_layers=2, seed=seed))
+    return out
+
+
+@pytest.mark.parametrize("wl", small_cases() + reseeded_cases(), ids=lambda w: w.name)
 def test_end_to_end_with_teacher_forcing(wl):
     ctx = make_ctx(wl)
     buf = P.GpuBuffers(wl)

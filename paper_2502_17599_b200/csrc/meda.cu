@@ -17,6 +17,7 @@
 #include "group_reduce.cuh"
 #include "merge_generic.cuh"
 #include "nearest_sm100.cuh"
+#include "nearest_small_sm100.cuh"
 #include "prompt_scores_sm100.cuh"
 #include "select.cuh"
 
@@ -469,6 +470,21 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
     LaunchScope scope(ctx, MEDA_K_NEAREST, st);
     nearest_kernel<<<std::min(items, ctx->sm_count), kNtThreads, NearestSmem::alloc, st>>>(map_kc, prm, ctx->ws.status);
   }
+  // The budget stays on the device, so both kernels are enqueued and the layer's S decides on the device which
+  // of them works: a layer with few slots streams the key cache in row order instead.
+  CUtensorMap map_k, map_kc128;
+  if (!make_rows_map(ctx, &map_k, k, n, c.n_kv_heads, n, 128) ||
+      !make_rows_map(ctx, &map_kc128, ctx->ws.kc, ctx->kc_rows, c.n_kv_heads, ctx->kc_rows, 128))
+    return MEDA_ERR_CUDA;
+  {
+    NearestSmallPolicy::Params prm{ctx->ws.inv_norm, budget_row, idx_conserved, target, n, c.n_kv_heads, cap,
+                                   ctx->inv_stride, (n + 255) / 256};
+    const int items = prm.row_blocks * c.n_kv_heads;
+    LaunchScope scope(ctx, MEDA_K_NEAREST, st);
+    umma_stream_kernel<NearestSmallPolicy><<<std::min(items, ctx->sm_count), us_threads<NearestSmallPolicy>(),
+                                             StreamShared<NearestSmallPolicy>::alloc, st>>>(map_k, map_kc128, prm,
+                                                                                            ctx->ws.status);
+  }
   return launch_status();
 }
 
@@ -814,6 +830,9 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     }
     if (st == MEDA_OK && cudaFuncSetAttribute(nearest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)NearestSmem::alloc) != cudaSuccess)
+      st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<NearestSmallPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)StreamShared<NearestSmallPolicy>::alloc) != cudaSuccess)
       st = MEDA_ERR_CUDA;
     if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<PromptStatsPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)StreamShared<PromptStatsPolicy>::alloc) != cudaSuccess)

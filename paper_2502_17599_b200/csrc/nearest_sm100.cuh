@@ -37,6 +37,9 @@ constexpr uint32_t kNtStageBytes = 2 * kNtHalf;
 constexpr uint32_t kNtTmemCols = 512;
 constexpr uint32_t kNtAccBase = 128;                    // first accumulator column
 constexpr uint32_t kNtAccBuf = 2 * kNtTileN;            // columns per accumulator buffer
+// Layers that keep at most this many slots take the streaming kernel of nearest_small_sm100.cuh instead: with
+// one or a few slot tiles per row block, loading the rows by index into tensor memory dominates here.
+constexpr int kNearestSmallMaxS = 1024;
 
 // Gathers the conserved keys of every KV head into a dense operand and computes their inverse
 // norms: kc[g][s][:] = k[g][c_s][:], inv_norm[g][s] = 1 / max(|k[g][c_s]|, eps).  One warp per slot.
@@ -160,7 +163,7 @@ nearest_kernel(const __grid_constant__ CUtensorMap map_kc, const NearestParams p
 
   // work of this launch, from the layer's budget row (uniform over the grid)
   const int S = min(p.budget_row[0], p.cap);
-  if (S <= 0 || S >= p.n) return;                                  // nothing to merge
+  if (S <= kNearestSmallMaxS || S >= p.n) return;                  // nothing to merge, or the streaming kernel's layer
   // only the less-important rows are swept: a row block is 256 consecutive entries of the head's list
   const int n_less = p.n - S;
   const int m_blocks = (n_less + 255) / 256;

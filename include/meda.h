@@ -255,6 +255,7 @@ enum {
   MEDA_K_SELECT,         /* radix select + compaction */
   MEDA_K_PREP,           /* conserved-key gather and inverse norms */
   MEDA_K_NEAREST,        /* similarity contraction + arg-max */
+  MEDA_K_NEAREST_SMALL,  /* the same step by the streaming kernel that layers with few kept slots take */
   MEDA_K_GROUP,          /* grouping of the less-important rows by target slot */
   MEDA_K_REDUCE,         /* segmented average */
   MEDA_K_DECODE,         /* decoding-step attention over a cache */

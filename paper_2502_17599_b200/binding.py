@@ -24,7 +24,8 @@ MEDA_ERR_CUDA = -5
 MEDA_ERR_UNSUPPORTED = -6
 MEDA_ERR_TIMEOUT = -7
 
-N_KERNEL_CLASSES = 11
+N_KERNEL_CLASSES = 12
+NEAREST_SMALL_MAX_S = 384   # kNearestSmallMaxS: layers keeping at most this many slots take the streaming arg-max kernel
 
 MEDA_BF16 = 0
 MEDA_F32 = 1

@@ -480,7 +480,7 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
     NearestSmallPolicy::Params prm{ctx->ws.inv_norm, budget_row, idx_conserved, target, n, c.n_kv_heads, cap,
                                    ctx->inv_stride, (n + 255) / 256};
     const int items = prm.row_blocks * c.n_kv_heads;
-    LaunchScope scope(ctx, MEDA_K_NEAREST, st);
+    LaunchScope scope(ctx, MEDA_K_NEAREST_SMALL, st);
     umma_stream_kernel<NearestSmallPolicy><<<std::min(items, ctx->sm_count), us_threads<NearestSmallPolicy>(),
                                              StreamShared<NearestSmallPolicy>::alloc, st>>>(map_k, map_kc128, prm,
                                                                                             ctx->ws.status);
@@ -877,7 +877,8 @@ int64_t meda_launch_count(const meda_ctx* ctx) { return ctx ? ctx->launches : 0;
 
 const char* meda_kernel_class_name(int32_t kernel_class) {
   static const char* const names[MEDA_K_CLASSES] = {"stats", "stats_combine", "sweep", "entropy_final", "allocate",
-                                                    "select", "prep", "nearest", "group", "reduce", "decode"};
+                                                    "select", "prep", "nearest", "nearest_small", "group", "reduce",
+                                                    "decode"};
   return kernel_class >= 0 && kernel_class < MEDA_K_CLASSES ? names[kernel_class] : nullptr;
 }
 

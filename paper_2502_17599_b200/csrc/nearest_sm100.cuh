@@ -38,8 +38,10 @@ constexpr uint32_t kNtTmemCols = 512;
 constexpr uint32_t kNtAccBase = 128;                    // first accumulator column
 constexpr uint32_t kNtAccBuf = 2 * kNtTileN;            // columns per accumulator buffer
 // Layers that keep at most this many slots take the streaming kernel of nearest_small_sm100.cuh instead: with
-// one or a few slot tiles per row block, loading the rows by index into tensor memory dominates here.
-constexpr int kNearestSmallMaxS = 1024;
+// one to three slot tiles per row block, loading the rows by index into tensor memory dominates here.  Beyond
+// that the streaming kernel loses: its UMMAs read both operands from shared memory (measured break-even
+// between 350 and 600 slots, depending on the number of KV heads).
+constexpr int kNearestSmallMaxS = 384;
 
 // Gathers the conserved keys of every KV head into a dense operand and computes their inverse
 // norms: kc[g][s][:] = k[g][c_s][:], inv_norm[g][s] = 1 / max(|k[g][c_s]|, eps).  One warp per slot.

@@ -23,13 +23,34 @@ constexpr int kSegChunk = 128;        // sorted rows walked by one warp
 constexpr int kSegWarps = 2;         // small blocks: more of them fit, also beside a resident tensor-core block
 
 // ---- stable radix pass: histogram, scan, scatter ----------------------------------------------
-// table[g][bin][block] <- number of keys of block `block` whose digit is `bin`.
+// The keys are slots < S, so the pass over the digit at `shift` orders nothing when S <= 2^shift: its three
+// kernels return at once (the host enqueues the passes the prompt length may need; the layer's budget is only
+// known on the device) and the consumer picks the buffer the last executed pass wrote.
+__device__ __forceinline__ bool sort_pass_needed(int S, int shift) { return shift == 0 || S > (1 << shift); }
+// Passes executed for a layer with S slots, of the `max_passes` the host enqueued.
+__device__ __forceinline__ int sort_passes_done(int S, int max_passes) {
+  int done = 1;
+  while (done < max_passes && sort_pass_needed(S, done * kSortBits)) ++done;
+  return done;
+}
+
+// table[g][bin][block] <- number of keys of block `block` whose digit is `bin`.  The first pass also clears
+// the per-slot segment bounds of the layer (slots without members must read as empty).
 __global__ void __launch_bounds__(kSortWarps * 32)
 sort_hist_kernel(const int32_t* __restrict__ keys, const int32_t* __restrict__ budget_row, int32_t* __restrict__ table,
-                 int n, int cap, int shift, int n_blocks) {
+                 int n, int cap, int shift, int n_blocks, int32_t* __restrict__ seg_start,
+                 int32_t* __restrict__ seg_end) {
   __shared__ int cnt[kSortBins];
   const int g = blockIdx.y, blk = blockIdx.x;
-  const int n_less = n - min(budget_row[0], cap);
+  const int S = min(budget_row[0], cap);
+  if (!sort_pass_needed(S, shift)) return;
+  const int n_less = n - S;
+  if (shift == 0) {
+    for (int s = blk * blockDim.x + threadIdx.x; s < S; s += gridDim.x * blockDim.x) {
+      seg_start[(size_t)g * n + s] = 0;
+      seg_end[(size_t)g * n + s] = 0;
+    }
+  }
   for (int b = threadIdx.x; b < kSortBins; b += blockDim.x) cnt[b] = 0;
   __syncthreads();
   const int32_t* kg = keys + (size_t)g * n;
@@ -46,8 +67,10 @@ sort_hist_kernel(const int32_t* __restrict__ keys, const int32_t* __restrict__ b
 // In-place exclusive prefix sum of each head's table in (bin, chunk) order.  One block per head;
 // `len` is a multiple of 4096 (the chunk count is padded to a multiple of 8), so every thread owns
 // a run of len / 1024 entries that is a whole number of 16-byte vectors.
-__global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ table, int len) {
+__global__ void __launch_bounds__(1024)
+sort_scan_kernel(int32_t* __restrict__ table, int len, const int32_t* __restrict__ budget_row, int cap, int shift) {
   __shared__ int warp_sums[32];
+  if (!sort_pass_needed(min(budget_row[0], cap), shift)) return;
   int4* t = reinterpret_cast<int4*>(table + (size_t)blockIdx.x * len);
   const int per = len / 4096;                         // vectors per thread
   const int begin = (int)threadIdx.x * per;
@@ -100,7 +123,9 @@ sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restri
                     int n_blocks) {
   __shared__ int cnt[kSortWarps][kSortBins];
   const int g = blockIdx.y, blk = blockIdx.x, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int n_less = n - min(budget_row[0], cap);
+  const int S_layer = min(budget_row[0], cap);
+  if (!sort_pass_needed(S_layer, shift)) return;
+  const int n_less = n - S_layer;
   if (blk * kSortBlockItems >= n_less) return;            // uniform over the block
   const int32_t* kg = keys_in + (size_t)g * n;
   const int32_t* rg = rows_in + (size_t)g * n;
@@ -212,8 +237,9 @@ __device__ __forceinline__ void store_row(T* p, int lane, const float (&x)[E], f
 // as many warps keep rows in flight; the z = 0 warps also record segment bounds and counts.
 template <typename T, int D>
 __global__ void __launch_bounds__(kSegWarps * 32, 9)
-seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ keys,
-                  const int32_t* __restrict__ rows, const int32_t* __restrict__ idx_conserved,
+seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ keys_a,
+                  const int32_t* __restrict__ rows_a, const int32_t* __restrict__ keys_b,
+                  const int32_t* __restrict__ rows_b, int max_passes, const int32_t* __restrict__ idx_conserved,
                   const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,
                   int32_t* __restrict__ counts, int32_t* __restrict__ seg_start, int32_t* __restrict__ seg_end,
                   float* __restrict__ carry, int32_t* __restrict__ carry_cnt, int n, int cap, int n_chunks) {
@@ -227,8 +253,10 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
   const int q0 = chunk * kSegChunk;
   if (q0 >= n_less) return;
   const int q1 = min(q0 + kSegChunk, n_less);
-  const int32_t* kg = keys + (size_t)g * n;
-  const int32_t* rg = rows + (size_t)g * n;
+  // the grouped list is in the buffer the last executed sort pass wrote: pass p writes buffer p % 2
+  const bool in_b = ((sort_passes_done(S, max_passes) - 1) & 1) != 0;
+  const int32_t* kg = (in_b ? keys_b : keys_a) + (size_t)g * n;
+  const int32_t* rg = (in_b ? rows_b : rows_a) + (size_t)g * n;
   const T* x_g = (tensor == 0 ? k : v) + (size_t)g * n * D;
   T* out_g = (tensor == 0 ? k_out : v_out) + (size_t)g * cap * D;
   const int32_t* cons = idx_conserved + (size_t)g * cap;
@@ -366,17 +394,6 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
     }
     store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)(members + 1));
     if (tensor == 0 && lane == 0) counts[(size_t)g * cap + slot] = members + 1;
-  }
-}
-
-// Clears the per-slot segment bounds of one layer (slots without members must read as empty).
-__global__ void clear_segments_kernel(int32_t* __restrict__ seg_start, int32_t* __restrict__ seg_end,
-                                      const int32_t* __restrict__ budget_row, int n, int cap) {
-  const int g = blockIdx.y;
-  const int S = min(budget_row[0], cap);
-  for (int s = blockIdx.x * blockDim.x + threadIdx.x; s < S; s += gridDim.x * blockDim.x) {
-    seg_start[(size_t)g * n + s] = 0;
-    seg_end[(size_t)g * n + s] = 0;
   }
 }
 

@@ -491,15 +491,16 @@ meda_status launch_nearest_fast(meda_ctx* ctx, const void* k, const int32_t* bud
 // Grouping sort + segmented average (Eq. 12) for any dtype / head_dim.
 template <typename T, int D>
 void launch_seg_kernels(meda_ctx* ctx, const void* k, const void* v, const int32_t* budget_row,
-                        const int32_t* idx_conserved, const int32_t* keys, const int32_t* rows, void* k_out,
-                        void* v_out, int32_t* counts, int32_t cap, int evict, cudaStream_t st) {
+                        const int32_t* idx_conserved, void* k_out, void* v_out, int32_t* counts, int32_t cap,
+                        int evict, cudaStream_t st) {
   const meda_config& c = ctx->cfg;
   const int n = c.n_tokens;
   const int max_slots = std::min(cap, n);
   if (!evict) {
     LaunchScope scope(ctx, MEDA_K_REDUCE, st);
     seg_reduce_kernel<T, D><<<dim3((ctx->seg_chunks + kSegWarps - 1) / kSegWarps, c.n_kv_heads, 2), kSegWarps * 32, 0, st>>>(
-        static_cast<const T*>(k), static_cast<const T*>(v), keys, rows, idx_conserved, budget_row,
+        static_cast<const T*>(k), static_cast<const T*>(v), ctx->ws.sort_keys[0], ctx->ws.sort_rows[0],
+        ctx->ws.sort_keys[1], ctx->ws.sort_rows[1], ctx->sort_passes, idx_conserved, budget_row,
         static_cast<T*>(k_out), static_cast<T*>(v_out), counts, ctx->ws.seg_start, ctx->ws.seg_end, ctx->ws.carry,
         ctx->ws.carry_cnt, n, cap, ctx->seg_chunks);
   }
@@ -521,11 +522,6 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
   const int32_t* keys = target;
   const int32_t* rows = idx_less;
   if (!evict) {
-    {
-      LaunchScope scope(ctx, MEDA_K_GROUP, st);
-      clear_segments_kernel<<<dim3(slot_blocks(ctx, max_slots, 256, c.n_kv_heads), c.n_kv_heads), 256, 0, st>>>(ctx->ws.seg_start,
-                                                                                       ctx->ws.seg_end, budget_row, n, cap);
-    }
     const dim3 grid(ctx->sort_chunks, c.n_kv_heads);
     for (int pass = 0; pass < ctx->sort_passes; ++pass) {
       int32_t* ko = ctx->ws.sort_keys[pass & 1];
@@ -534,11 +530,12 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
       {
         LaunchScope scope(ctx, MEDA_K_GROUP, st);
         sort_hist_kernel<<<grid, kSortWarps * 32, 0, st>>>(keys, budget_row, ctx->ws.sort_table, n, cap, shift,
-                                                           ctx->sort_chunks);
+                                                           ctx->sort_chunks, ctx->ws.seg_start, ctx->ws.seg_end);
       }
       {
         LaunchScope scope(ctx, MEDA_K_GROUP, st);
-        sort_scan_kernel<<<c.n_kv_heads, 1024, 0, st>>>(ctx->ws.sort_table, kSortBins * ctx->sort_chunks);
+        sort_scan_kernel<<<c.n_kv_heads, 1024, 0, st>>>(ctx->ws.sort_table, kSortBins * ctx->sort_chunks, budget_row,
+                                                        cap, shift);
       }
       {
         LaunchScope scope(ctx, MEDA_K_GROUP, st);
@@ -550,9 +547,9 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
     }
   }
   switch (c.head_dim) {
-    case 64: launch_seg_kernels<T, 64>(ctx, k, v, budget_row, idx_conserved, keys, rows, k_out, v_out, counts, cap, evict, st); break;
-    case 128: launch_seg_kernels<T, 128>(ctx, k, v, budget_row, idx_conserved, keys, rows, k_out, v_out, counts, cap, evict, st); break;
-    default: launch_seg_kernels<T, 256>(ctx, k, v, budget_row, idx_conserved, keys, rows, k_out, v_out, counts, cap, evict, st); break;
+    case 64: launch_seg_kernels<T, 64>(ctx, k, v, budget_row, idx_conserved, k_out, v_out, counts, cap, evict, st); break;
+    case 128: launch_seg_kernels<T, 128>(ctx, k, v, budget_row, idx_conserved, k_out, v_out, counts, cap, evict, st); break;
+    default: launch_seg_kernels<T, 256>(ctx, k, v, budget_row, idx_conserved, k_out, v_out, counts, cap, evict, st); break;
   }
   return launch_status();
 }

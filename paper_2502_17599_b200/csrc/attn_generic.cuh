@@ -277,6 +277,8 @@ __global__ void entropy_finalize_kernel(const float* __restrict__ ent_partial, i
                                         const float* __restrict__ row_stats, int w, float* __restrict__ entropy_out,
                                         int accumulate = 0) {
   __shared__ double red[256];
+  // window rows that see a key of the subset (head 0's normaliser tells): one row per thread, w <= 128
+  const int rows = __syncthreads_count((int)threadIdx.x < w && row_stats[threadIdx.x * 4 + 3] > 0.f);
   double acc = 0.0;
   for (int e = threadIdx.x; e < n_partials; e += blockDim.x) acc += (double)ent_partial[e];
   red[threadIdx.x] = acc;
@@ -286,8 +288,6 @@ __global__ void entropy_finalize_kernel(const float* __restrict__ ent_partial, i
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    int rows = 0;
-    for (int i = 0; i < w; ++i) rows += (row_stats[i * 4 + 3] > 0.f) ? 1 : 0;   // head 0
     const float term = rows > 0 ? (float)(-red[0] / (double)rows) : 0.f;
     *entropy_out = accumulate ? *entropy_out + term : term;      // E_CM = (-E_TV) + (-E_VT), Eq. 6
   }

@@ -768,11 +768,22 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   ctx->fast_attn = ctx->fast && (c.window == 32 || c.window == 64) && ctx->group * c.window <= kSweepMaxCols;
   ctx->ent_slots = std::max(generic_tiles(c.n_tokens), ((c.n_tokens + 255) / 256) * kUsEpilogueWarps);
   {
-    // key chunks of the tensor-core normaliser sweep: about two items per SM
+    // Key chunks of the tensor-core normaliser sweep.  An item = (KV head, row block, key chunk); the grid is
+    // one block per SM, so a launch takes ceil(items / SMs) waves of (tiles per chunk + about 1.5 tiles of
+    // per-item overhead: resident block reload, pipeline refill).  Take the chunk count with the cheapest
+    // estimate, at most four waves.
     const int tiles = (c.n_tokens + 127) / 128;
     const int row_blocks = (ctx->group * c.window + 255) / 256;
-    int want = std::max(1, (2 * ctx->sm_count) / std::max(1, c.n_kv_heads * row_blocks));
-    want = std::min(want, tiles);
+    const int per_chunk_items = std::max(1, c.n_kv_heads * row_blocks);
+    int want = 1;
+    double best = 1e300;
+    for (int cand = 1; cand <= tiles && cand * per_chunk_items <= 4 * ctx->sm_count; ++cand) {
+      const int tpc = (tiles + cand - 1) / cand;
+      const int chunks = (tiles + tpc - 1) / tpc;
+      const int waves = (chunks * per_chunk_items + ctx->sm_count - 1) / ctx->sm_count;
+      const double cost = waves * (tpc + 1.5);
+      if (cost < best) { best = cost; want = cand; }
+    }
     ctx->stats_tiles_per_chunk = (tiles + want - 1) / want;
     ctx->stats_chunks = (tiles + ctx->stats_tiles_per_chunk - 1) / ctx->stats_tiles_per_chunk;
   }

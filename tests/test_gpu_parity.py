@@ -229,6 +229,40 @@ def test_merge_kv_against_oracle_sets(wl, merge_mode):
     ctx.close()
 
 
+@pytest.mark.parametrize("S", [96, 97, 384, 385, 512, 513, 1024])
+def test_merge_at_the_budgets_where_the_kernels_switch(S):
+    """The layer's slot count decides on the device which arg-max kernel works (streaming up to 384 slots,
+    row-gathering above) and how many passes the grouping sort executes (one up to 512 slots): both sides of
+    each switch, and of a slot-tile border, on a prompt of 2,857 tokens, against the oracle."""
+    wl = W.small_variant("switch_2857", spans=W._spans((37, 0), (45 * 61, 1), (75, 0)), window=32, seed=13)
+    n = wl.n_tokens
+    ctx = make_ctx(wl)
+    buf = P.GpuBuffers(wl)
+    mod = wl.modality().numpy()
+    (q, k, v), (qh, kh, vh) = P.layer_inputs(wl, 0, "cuda")
+    a_s = O.window_scores(qh, kh)
+    M = (3 * S) // 4
+    N = S - M
+    sets = [O.select_topk(a_s[g], mod, M, N) for g in range(wl.n_kv_heads)]
+    for g, (c, ls) in enumerate(sets):
+        buf.idx_c[g, :S] = torch.from_numpy(c.astype(np.int32)).cuda()
+        buf.idx_less[g, : n - S] = torch.from_numpy(ls.astype(np.int32)).cuda()
+    budgets = torch.tensor([[S, M, N]] * wl.n_layers, dtype=torch.int32, device="cuda")
+    buf.k_out.fill_(7.0)
+    buf.target.fill_(-1)
+    ctx.merge_kv(0, k, v, budgets, buf.idx_c, buf.idx_less, buf.k_out, buf.v_out, buf.counts, buf.target, buf.cap)
+    ctx.check()
+    for g, (c, ls) in enumerate(sets):
+        tgt = buf.target[g, : n - S].cpu().numpy()
+        assert (buf.target[g, n - S:] == -1).all()       # nothing written past the less-important list
+        P.compare_targets(tgt, kh[g], c, ls)
+        P.compare_merged(P.np64(buf.k_out[g, :S]), P.np64(buf.v_out[g, :S]), buf.counts[g, :S].cpu().numpy(),
+                         kh[g], vh[g], c, ls, tgt, wl.dtype)
+        assert int(buf.counts[g, :S].sum()) == n
+        assert (buf.k_out[g, S:] == 7.0).all()
+    ctx.close()
+
+
 def test_merge_special_cases_on_device():
     """Duplicate keys merge into their twin; a single conserved slot becomes the arithmetic mean."""
     wl = W.small_variant("special", n_layers=1, frame_rho=0.0, salient_frac=0.0)

@@ -65,14 +65,17 @@ class CompressionPass:
             ev.record(s)
             main.wait_event(ev)
 
-    def run(self, q_layers, k_layers, v_layers, stream=None, single_stream=False, qk_ready=None, v_ready=None):
+    def run(self, q_layers, k_layers, v_layers, stream=None, single_stream=False, qk_ready=None, v_ready=None,
+            budgets_done=None, layer_done=None):
         """Enqueues the whole pass.  Inputs are lists of per-layer device tensors; results stay on the
         device in this object's buffers.  The work is ordered after what `stream` (default: torch's
         current stream) holds and `stream` waits for all of it.  With `single_stream` everything goes to
         `stream` through the first context (used when every launch is timed on its own).  `qk_ready` /
         `v_ready`: optional per-layer events after which a layer's (queries, keys) / values are in
         place (copies still in flight on another stream): phase A of a layer waits for the first,
-        phase B for the second."""
+        phase B for the second.  `budgets_done` (an event) is recorded once the budgets are written,
+        `layer_done[l]` (events) once layer l's compressed cache is: a caller can start copying results
+        out while later layers are still being compressed."""
         L = self.wl.n_layers
         main = stream if stream is not None else torch.cuda.current_stream()
         if single_stream or not self.streams:
@@ -88,6 +91,8 @@ class CompressionPass:
         if len(lanes) > 1:
             self._join(main)
         self.ctx.allocate_budgets(self.entropy, self.budgets, main)      # Eq. 7 needs every layer's entropy
+        if budgets_done is not None:
+            budgets_done.record(main)
         if len(lanes) > 1:
             self._fork(main)
         for l in range(L):
@@ -96,6 +101,8 @@ class CompressionPass:
                 s.wait_event(v_ready[l])
             c.compress_layer(l, k_layers[l], v_layers[l], self.scores[l], self.budgets, self.k_out[l], self.v_out[l],
                              self.counts[l], self.idx_c[l], self.cap, s)
+            if layer_done is not None:
+                layer_done[l].record(s)
         if len(lanes) > 1:
             self._join(main)
 
@@ -148,16 +155,29 @@ class CompressionPass:
                 ev = torch.cuda.Event()
                 ev.record(cs)
                 v_ready.append(ev)
-        self.run(staging["q"], staging["k"], staging["v"], qk_ready=qk_ready, v_ready=v_ready)
-        out_host["budgets"].copy_(self.budgets, non_blocking=True)
-        torch.cuda.current_stream().synchronize()      # the live row counts decide what comes back
-        d2h = self.budgets.numel() * 4
-        for l in range(L):
-            s = int(out_host["budgets"][l, 0])
-            for name, src in (("k", self.k_out), ("v", self.v_out), ("counts", self.counts), ("idx", self.idx_c)):
-                out_host[name][l].copy_(src[l][:, :s], non_blocking=True)
-                d2h += src[l][:, :s].numel() * src.element_size()
-        torch.cuda.current_stream().synchronize()
+        budgets_done = torch.cuda.Event()
+        layer_done = [torch.cuda.Event() for _ in range(L)]
+        self.run(staging["q"], staging["k"], staging["v"], qk_ready=qk_ready, v_ready=v_ready,
+                 budgets_done=budgets_done, layer_done=layer_done)
+        # Results leave on a third stream: the budgets as soon as they exist (the live row counts decide
+        # what comes back), then each layer's compacted cache as soon as that layer is done, while the
+        # values of later layers are still arriving (the link carries both directions at once).
+        if not hasattr(self, "_down_stream"):
+            self._down_stream = torch.cuda.Stream(device=self.device)
+        ds = self._down_stream
+        with torch.cuda.stream(ds):
+            ds.wait_event(budgets_done)
+            out_host["budgets"].copy_(self.budgets, non_blocking=True)
+            ds.synchronize()
+            d2h = self.budgets.numel() * 4
+            for l in range(L):
+                s = int(out_host["budgets"][l, 0])
+                ds.wait_event(layer_done[l])
+                for name, src in (("k", self.k_out), ("v", self.v_out), ("counts", self.counts), ("idx", self.idx_c)):
+                    out_host[name][l].copy_(src[l][:, :s], non_blocking=True)
+                    d2h += src[l][:, :s].numel() * src.element_size()
+        main.wait_stream(ds)
+        main.synchronize()
         return h2d, d2h
 
     def alloc_host_outputs(self):

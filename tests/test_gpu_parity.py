@@ -493,3 +493,43 @@ def test_degenerate_sizes_on_the_tensor_core_paths():
             assert torch.equal(buf.k_out[:, :n], k) and torch.equal(buf.v_out[:, :n], v) and (buf.counts[:, :n] == 1).all()
         assert (buf.k_out[:, S:] == 7.0).all()
     ctx.close()
+
+
+@pytest.mark.parametrize("wl", [W.small_variant("host_path_tc", window=32, seed=14), W.WORKLOADS["tiny"]],
+                         ids=lambda w: w.name)
+def test_pass_from_pinned_host_buffers_returns_what_the_device_pass_holds(wl):
+    """The host-buffer variant of the whole pass (inputs copied in layer by layer while earlier layers are
+    processed, results copied out layer by layer while later layers are compressed) gives the same bits as
+    the pass over device-resident inputs, and reports the bytes it moved."""
+    from paper_2502_17599_b200.pipeline import CompressionPass
+    L = wl.n_layers
+    qs, ks, vs = [], [], []
+    for l in range(L):
+        q, k, v = W.make_layer(wl, l, "cuda")
+        qs.append(q); ks.append(k); vs.append(v)
+    cp = CompressionPass(wl)
+    cp.run(qs, ks, vs)
+    cp.check()
+    budgets = cp.budgets.cpu()
+    want = {name: [src[l][:, : int(budgets[l, 0])].cpu() for l in range(L)]
+            for name, src in (("k", cp.k_out), ("v", cp.v_out), ("counts", cp.counts), ("idx", cp.idx_c))}
+    q_h = [t.cpu().pin_memory() for t in qs]
+    k_h = [t.cpu().pin_memory() for t in ks]
+    v_h = [t.cpu().pin_memory() for t in vs]
+    staging = {"q": [torch.zeros_like(t) for t in qs], "k": [torch.zeros_like(t) for t in ks],
+               "v": [torch.zeros_like(t) for t in vs]}
+    out_host = cp.alloc_host_outputs()
+    for _ in range(2):
+        for name in ("k", "v", "counts", "idx"):
+            for t in out_host[name]:
+                t.zero_()
+        h2d, d2h = cp.run_from_host(q_h, k_h, v_h, staging, out_host)
+        cp.check()
+        assert torch.equal(out_host["budgets"], budgets)
+        for name in ("k", "v", "counts", "idx"):
+            for l in range(L):
+                assert torch.equal(out_host[name][l], want[name][l]), (name, l)
+        assert h2d == sum(t.numel() * t.element_size() for t in q_h + k_h + v_h)
+        assert d2h == budgets.numel() * 4 + sum(t.numel() * t.element_size()
+                                                for name in ("k", "v", "counts", "idx") for t in out_host[name])
+    cp.close()

@@ -860,8 +860,11 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     st = c.dtype == MEDA_F32 ? set_generic_attrs<float>() : set_generic_attrs<__nv_bfloat16>();
   }
   // selection: one cluster per KV head while a head's keys fit the cluster's shared memory
-  ctx->select_cluster = select_cluster_smem(c.n_tokens).total <= kMaxDynSmem;
-  if (st == MEDA_OK && ctx->select_cluster) st = raise_dyn_smem(select_topk_cluster_kernel);
+  ctx->select_cluster = select_cluster_size(c.n_tokens, c.n_kv_heads, ctx->sm_count, kMaxDynSmem);
+  if (st == MEDA_OK && ctx->select_cluster == 8) st = raise_dyn_smem(select_topk_cluster_kernel<8>);
+  if (st == MEDA_OK && ctx->select_cluster == 4) st = raise_dyn_smem(select_topk_cluster_kernel<4>);
+  if (st == MEDA_OK && ctx->select_cluster == 2) st = raise_dyn_smem(select_topk_cluster_kernel<2>);
+  if (st == MEDA_OK && ctx->select_cluster == 1) st = raise_dyn_smem(select_topk_cluster_kernel<1>);
   if (st != MEDA_OK) {
     free_workspace(ws);
     delete ctx;
@@ -1019,11 +1022,19 @@ meda_status meda_select_topk(meda_ctx* ctx, int32_t layer, const float* scores, 
   if (out_capacity < 1) return MEDA_ERR_WORKSPACE;
   const meda_config& c = ctx->cfg;
   LaunchScope scope(ctx, MEDA_K_SELECT, as_stream(stream));
-  if (ctx->select_cluster)
-    select_topk_cluster_kernel<<<kSelClusterSize * c.n_kv_heads, kSelThreads, select_cluster_smem(c.n_tokens).total,
-                                 as_stream(stream)>>>(scores, ctx->ws.modality, budgets + (size_t)layer * 3,
-                                                      idx_conserved, idx_less, c.n_tokens, out_capacity, ctx->ws.status);
-  else
+  if (ctx->select_cluster) {
+    const int cs = ctx->select_cluster;
+    const int smem = select_cluster_smem(c.n_tokens, cs).total;
+    const int32_t* row = budgets + (size_t)layer * 3;
+#define MEDA_LAUNCH_SELECT(C)                                                                                  \
+  select_topk_cluster_kernel<C><<<C * c.n_kv_heads, kSelThreads, smem, as_stream(stream)>>>(                    \
+      scores, ctx->ws.modality, row, idx_conserved, idx_less, c.n_tokens, out_capacity, ctx->ws.status)
+    if (cs == 8) MEDA_LAUNCH_SELECT(8);
+    else if (cs == 4) MEDA_LAUNCH_SELECT(4);
+    else if (cs == 2) MEDA_LAUNCH_SELECT(2);
+    else MEDA_LAUNCH_SELECT(1);
+#undef MEDA_LAUNCH_SELECT
+  } else
     select_topk_kernel<<<c.n_kv_heads, kSelThreads, 0, as_stream(stream)>>>(
         scores, ctx->ws.modality, budgets + (size_t)layer * 3, idx_conserved, idx_less, c.n_tokens, out_capacity,
         ctx->ws.status);

@@ -69,7 +69,7 @@ struct meda_ctx {
   int sort_passes = 1;    // 9-bit digit passes needed to order slots < n_tokens
   bool fast = false;      // bf16 with head_dim 128: tensor-core kernels are used
   bool fast_attn = false; // ... and window 32 or 64: phase A runs on the tensor cores too
-  bool select_cluster = false;   // selection runs as one thread-block cluster per KV head
+  int select_cluster = 0;        // blocks per thread-block cluster (one cluster per KV head) of the selection; 0: single-block kernel
   int stats_chunks = 0;   // key chunks of the tensor-core normaliser sweep
   int stats_tiles_per_chunk = 0;
   void* encode_tiled = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime

@@ -118,13 +118,15 @@ select_topk_kernel(const float* __restrict__ scores, const uint8_t* __restrict__
 
 // ---------------------------------------------------------------------------------------------
 // The same selection with one thread-block cluster per KV head, for sequences whose keys fit the
-// cluster's shared memory: the 8 blocks of a cluster each stage one eighth of the head's scores
+// cluster's shared memory: the C blocks of a cluster each stage one C-th of the head's scores
 // as 32-bit sort keys, so the radix passes read shared memory only; digit histograms are combined
 // across the cluster through distributed shared memory, and the hardware cluster barrier is the
 // only synchronisation between blocks.  Same ranking, same tie-break, same outputs as the
-// single-block kernel above.
+// single-block kernel above.  C is 8 for long prompts and smaller (4, 2, 1) when an eighth of the
+// prompt would be less than one compaction step per block or when 8 blocks per head would need more
+// than one wave of the GPU (see select_cluster_size).
 // ---------------------------------------------------------------------------------------------
-constexpr int kSelClusterSize = 8;
+constexpr int kSelMaxClusterSize = 8;
 constexpr int kSelBins = 2048;                    // 11-bit digits: 11 + 11 + 10 bits of the score key
 constexpr int kSelPerThread = 4;                  // consecutive tokens per thread in the compaction
 
@@ -132,10 +134,10 @@ struct SelectClusterSmem {
   int chunk;          // tokens per block
   int keys_off, hist_off, total_off, misc_off, total;
 };
-__host__ __device__ inline SelectClusterSmem select_cluster_smem(int n) {
+__host__ __device__ inline SelectClusterSmem select_cluster_smem(int n, int cluster_size) {
   SelectClusterSmem L;
   const int step = kSelThreads * kSelPerThread;
-  L.chunk = ((n + kSelClusterSize - 1) / kSelClusterSize + step - 1) / step * step;
+  L.chunk = ((n + cluster_size - 1) / cluster_size + step - 1) / step * step;
   int off = 0;
   L.keys_off = off;  off += L.chunk * 4;
   L.hist_off = off;  off += kSelBins * 4;
@@ -172,6 +174,19 @@ __device__ __forceinline__ int block_exclusive_sum(int v, int* scratch, int& tot
   return scratch[warp] + incl - v;
 }
 
+// Blocks per head: the largest of 8, 4, 2, 1 that gives every block at least one compaction step of tokens
+// and keeps all heads' clusters within one wave of `sm_count` blocks, as long as the keys of a block still
+// fit `smem_limit` bytes; 0 if even eight blocks per head do not fit (the single-block kernel then runs).
+inline int select_cluster_size(int n, int n_heads, int sm_count, int smem_limit) {
+  if (select_cluster_smem(n, kSelMaxClusterSize).total > smem_limit) return 0;
+  int c = kSelMaxClusterSize;
+  while (c > 1 && ((n + c - 1) / c < kSelThreads * kSelPerThread || n_heads * c > sm_count) &&
+         select_cluster_smem(n, c / 2).total <= smem_limit)
+    c /= 2;
+  return c;
+}
+
+template <int kSelClusterSize>
 __global__ void __cluster_dims__(kSelClusterSize, 1, 1) __launch_bounds__(kSelThreads)
 select_topk_cluster_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ modality,
                            const int32_t* __restrict__ budget_row, int32_t* __restrict__ idx_conserved,
@@ -179,7 +194,7 @@ select_topk_cluster_kernel(const float* __restrict__ scores, const uint8_t* __re
   namespace cg = cooperative_groups;
   extern __shared__ __align__(16) unsigned char sel_smem[];
   cg::cluster_group cluster = cg::this_cluster();
-  const SelectClusterSmem L = select_cluster_smem(n);
+  const SelectClusterSmem L = select_cluster_smem(n, kSelClusterSize);
   unsigned int* keys = reinterpret_cast<unsigned int*>(sel_smem + L.keys_off);
   unsigned int* hist = reinterpret_cast<unsigned int*>(sel_smem + L.hist_off);
   unsigned int* total = reinterpret_cast<unsigned int*>(sel_smem + L.total_off);

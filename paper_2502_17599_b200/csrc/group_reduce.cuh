@@ -1,12 +1,14 @@
 // Phase B, merge step 2 (Eq. 12): average every conserved row with the less-important rows
 // assigned to it, for keys and values, deterministically.
 //
-// The less-important rows are first grouped by target slot with a stable least-significant-digit
-// radix sort (9-bit digits; stability keeps the rows of a slot in ascending token order), so every
-// slot's members are contiguous and ordered.  Warps then walk fixed 128-row chunks of the sorted
-// list, summing in fp32 in list order; a slot whose members lie inside one chunk is finished on the
-// spot (own row first, then its members, one division, one rounding), pieces of slots that cross
-// chunk borders are parked as partial sums and added up in chunk order by a second small kernel.
+// All n token rows are first grouped by slot with a stable least-significant-digit radix sort
+// (9-bit digits): the list being sorted is the S kept rows (slot s, row c_s) followed by the n - S
+// less-important rows (their target slot, their row), so after the sort every slot's rows are
+// contiguous, the kept row first, then its members in ascending token order (stability).  Warps then
+// walk fixed 128-row chunks of the sorted list, summing in fp32 in list order: no row needs a
+// look-up of its own, every load address comes from the list.  A slot whose rows lie inside one chunk
+// is finished on the spot (one division, one rounding), pieces of slots that cross chunk borders are
+// parked as partial sums and added up in chunk order by a second small kernel.
 // No floating-point atomics anywhere: two runs give identical bits.
 #pragma once
 
@@ -34,30 +36,32 @@ __device__ __forceinline__ int sort_passes_done(int S, int max_passes) {
   return done;
 }
 
-// table[g][bin][block] <- number of keys of block `block` whose digit is `bin`.  The first pass also clears
-// the per-slot segment bounds of the layer (slots without members must read as empty).
+// Entry q of the list a pass reads.  The first pass (shift 0) reads the kept rows followed by the
+// less-important ones straight from the caller's arrays: q < S is (slot q, row idx_conserved[q]),
+// q >= S is (target[q - S], idx_less[q - S]); later passes read the previous pass's output.
+__device__ __forceinline__ int sort_key_at(const int32_t* __restrict__ keys, int q, int S, int shift) {
+  return shift == 0 ? (q < S ? q : keys[q - S]) : keys[q];
+}
+__device__ __forceinline__ int sort_row_at(const int32_t* __restrict__ rows, const int32_t* __restrict__ kept, int q,
+                                           int S, int shift) {
+  return shift == 0 ? (q < S ? kept[q] : rows[q - S]) : rows[q];
+}
+
+// table[g][bin][block] <- number of keys of block `block` whose digit is `bin`.
 __global__ void __launch_bounds__(kSortWarps * 32)
 sort_hist_kernel(const int32_t* __restrict__ keys, const int32_t* __restrict__ budget_row, int32_t* __restrict__ table,
-                 int n, int cap, int shift, int n_blocks, int32_t* __restrict__ seg_start,
-                 int32_t* __restrict__ seg_end) {
+                 int n, int cap, int shift, int n_blocks) {
   __shared__ int cnt[kSortBins];
   const int g = blockIdx.y, blk = blockIdx.x;
   const int S = min(budget_row[0], cap);
   if (!sort_pass_needed(S, shift)) return;
-  const int n_less = n - S;
-  if (shift == 0) {
-    for (int s = blk * blockDim.x + threadIdx.x; s < S; s += gridDim.x * blockDim.x) {
-      seg_start[(size_t)g * n + s] = 0;
-      seg_end[(size_t)g * n + s] = 0;
-    }
-  }
   for (int b = threadIdx.x; b < kSortBins; b += blockDim.x) cnt[b] = 0;
   __syncthreads();
   const int32_t* kg = keys + (size_t)g * n;
 #pragma unroll
   for (int r = 0; r < kSortBlockItems / (kSortWarps * 32); ++r) {
     const int q = blk * kSortBlockItems + r * (kSortWarps * 32) + (int)threadIdx.x;
-    if (q < n_less) atomicAdd(&cnt[(kg[q] >> shift) & (kSortBins - 1)], 1);
+    if (q < n) atomicAdd(&cnt[(sort_key_at(kg, q, S, shift) >> shift) & (kSortBins - 1)], 1);
   }
   __syncthreads();
   int32_t* tg = table + (size_t)g * kSortBins * n_blocks;
@@ -118,17 +122,18 @@ sort_scan_kernel(int32_t* __restrict__ table, int len, const int32_t* __restrict
 // warp ranks its elements in index order.
 __global__ void __launch_bounds__(kSortWarps * 32)
 sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restrict__ rows_in,
-                    const int32_t* __restrict__ budget_row, const int32_t* __restrict__ table,
+                    const int32_t* __restrict__ kept, const int32_t* __restrict__ budget_row,
+                    const int32_t* __restrict__ table,
                     int32_t* __restrict__ keys_out, int32_t* __restrict__ rows_out, int n, int cap, int shift,
                     int n_blocks) {
   __shared__ int cnt[kSortWarps][kSortBins];
   const int g = blockIdx.y, blk = blockIdx.x, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int S_layer = min(budget_row[0], cap);
   if (!sort_pass_needed(S_layer, shift)) return;
-  const int n_less = n - S_layer;
-  if (blk * kSortBlockItems >= n_less) return;            // uniform over the block
+  if (blk * kSortBlockItems >= n) return;                 // uniform over the block
   const int32_t* kg = keys_in + (size_t)g * n;
   const int32_t* rg = rows_in + (size_t)g * n;
+  const int32_t* kept_g = kept + (size_t)g * cap;
   int32_t* ko = keys_out + (size_t)g * n;
   int32_t* ro = rows_out + (size_t)g * n;
   const int q0 = blk * kSortBlockItems + warp * kSortWarpItems;
@@ -139,7 +144,7 @@ sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restri
 #pragma unroll
   for (int r = 0; r < kRounds; ++r) {
     const int q = q0 + r * 32 + lane;
-    key[r] = q < n_less ? kg[q] : -1;
+    key[r] = q < n ? sort_key_at(kg, q, S_layer, shift) : -1;
     if (key[r] >= 0) atomicAdd(&cnt[warp][(key[r] >> shift) & (kSortBins - 1)], 1);
   }
   __syncthreads();
@@ -160,7 +165,7 @@ sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restri
     const int q = q0 + r * 32 + lane;
     const bool valid = key[r] >= 0;
     const int digit = (key[r] >> shift) & (kSortBins - 1);
-    const int row = valid ? rg[q] : 0;
+    const int row = valid ? sort_row_at(rg, kept_g, q, S_layer, shift) : 0;
     const unsigned int peers = __match_any_sync(0xffffffffu, valid ? digit : kSortBins + lane);
     const int leader = __ffs(peers) - 1;
     int base = 0;
@@ -234,13 +239,13 @@ __device__ __forceinline__ void store_row(T* p, int lane, const float (&x)[E], f
 }
 
 // grid = (chunks / kSegWarps, heads, 2): blockIdx.z picks the tensor (0 keys, 1 values), so that twice
-// as many warps keep rows in flight; the z = 0 warps also record segment bounds and counts.
+// as many warps keep rows in flight; the z = 0 warps also record segment bounds and counts.  Every slot
+// has at least one row in the list (its kept row), so every slot's bounds get written.
 template <typename T, int D>
 __global__ void __launch_bounds__(kSegWarps * 32, 9)
 seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ keys_a,
                   const int32_t* __restrict__ rows_a, const int32_t* __restrict__ keys_b,
-                  const int32_t* __restrict__ rows_b, int max_passes, const int32_t* __restrict__ idx_conserved,
-                  const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,
+                  const int32_t* __restrict__ rows_b, int max_passes, const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,
                   int32_t* __restrict__ counts, int32_t* __restrict__ seg_start, int32_t* __restrict__ seg_end,
                   float* __restrict__ carry, int32_t* __restrict__ carry_cnt, int n, int cap, int n_chunks) {
   constexpr int E = D / 32;
@@ -249,17 +254,15 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
   const bool book = tensor == 0 && lane == 0;            // the one lane that writes bounds and counts
   const int chunk = blockIdx.x * kSegWarps + warp;
   const int S = min(budget_row[0], cap);
-  const int n_less = n - S;
   const int q0 = chunk * kSegChunk;
-  if (q0 >= n_less) return;
-  const int q1 = min(q0 + kSegChunk, n_less);
+  if (S <= 0 || q0 >= n) return;
+  const int q1 = min(q0 + kSegChunk, n);
   // the grouped list is in the buffer the last executed sort pass wrote: pass p writes buffer p % 2
   const bool in_b = ((sort_passes_done(S, max_passes) - 1) & 1) != 0;
   const int32_t* kg = (in_b ? keys_b : keys_a) + (size_t)g * n;
   const int32_t* rg = (in_b ? rows_b : rows_a) + (size_t)g * n;
   const T* x_g = (tensor == 0 ? k : v) + (size_t)g * n * D;
   T* out_g = (tensor == 0 ? k_out : v_out) + (size_t)g * cap * D;
-  const int32_t* cons = idx_conserved + (size_t)g * cap;
   int32_t* st = seg_start + (size_t)g * n;
   int32_t* en = seg_end + (size_t)g * n;
 
@@ -268,22 +271,18 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
   int cur = min(max(kg[q0], 0), S - 1);
   bool started_here = (q0 == 0) || (kg[q0 - 1] != kg[q0]);
 
+  // `members` counts the rows of the slot summed so far, the kept row included
   auto begin_segment = [&](int slot, bool fresh, int q) {
     members = 0;
-    if (fresh) {
-      const int own = min(max(cons[slot], 0), n - 1);
-      load_row<T, E>(x_g + (size_t)own * D, lane, acc);
-      if (book) st[slot] = q;
-    } else {
 #pragma unroll
-      for (int e = 0; e < E; ++e) acc[e] = 0.f;
-    }
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    if (fresh && book) st[slot] = q;
   };
   auto end_piece = [&](int slot, bool fresh, bool ended, int q_end) {
     if (ended && book) en[slot] = q_end;
     if (fresh && ended) {
-      store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)(members + 1));
-      if (book) counts[(size_t)g * cap + slot] = members + 1;
+      store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)members);
+      if (book) counts[(size_t)g * cap + slot] = members;
     } else {
       const int which = fresh ? 1 : 0;
       float* cp = carry_ptr<D>(carry, g, chunk, which, n_chunks) + tensor * D;
@@ -334,13 +333,13 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
       }
     }
   }
-  const bool ended = (q1 == n_less) || (min(max(kg[q1], 0), S - 1) != cur);
+  const bool ended = (q1 == n) || (min(max(kg[q1], 0), S - 1) != cur);
   end_piece(cur, started_here, ended, q1);
 }
 
-// One warp per (conserved slot, tensor): slots without members are copied, slots whose members span
-// several chunks get their parked pieces added in chunk order (loaded eight at a time, added one by
-// one); everything else was finished by the walker.  grid = (blocks, heads, 2).
+// One warp per (conserved slot, tensor): slots whose rows span several chunks get their parked pieces
+// added in chunk order (loaded eight at a time, added one by one); everything else was finished by the
+// walker.  Without merging (`evict`) the kept rows are copied.  grid = (blocks, heads, 2).
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ idx_conserved,
@@ -360,10 +359,12 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
     const int end = evict ? 0 : seg_end[(size_t)g * n + slot];
     float acc[E];
     int members = 0;
-    if (end <= start) {
+    if (evict) {
       const int own = min(max(idx_conserved[(size_t)g * cap + slot], 0), n - 1);
       load_row<T, E>(x_g + (size_t)own * D, lane, acc);
+      members = 1;
     } else {
+      if (end <= start) continue;                         // cannot happen: every slot has its kept row in the list
       const int c0 = start / kSegChunk, c1 = (end - 1) / kSegChunk;
       if (c0 == c1) continue;
       float* base = const_cast<float*>(carry);
@@ -392,8 +393,8 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
         }
       }
     }
-    store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)(members + 1));
-    if (tensor == 0 && lane == 0) counts[(size_t)g * cap + slot] = members + 1;
+    store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)members);
+    if (tensor == 0 && lane == 0) counts[(size_t)g * cap + slot] = members;
   }
 }
 

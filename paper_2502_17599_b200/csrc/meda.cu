@@ -500,7 +500,7 @@ void launch_seg_kernels(meda_ctx* ctx, const void* k, const void* v, const int32
     LaunchScope scope(ctx, MEDA_K_REDUCE, st);
     seg_reduce_kernel<T, D><<<dim3((ctx->seg_chunks + kSegWarps - 1) / kSegWarps, c.n_kv_heads, 2), kSegWarps * 32, 0, st>>>(
         static_cast<const T*>(k), static_cast<const T*>(v), ctx->ws.sort_keys[0], ctx->ws.sort_rows[0],
-        ctx->ws.sort_keys[1], ctx->ws.sort_rows[1], ctx->sort_passes, idx_conserved, budget_row,
+        ctx->ws.sort_keys[1], ctx->ws.sort_rows[1], ctx->sort_passes, budget_row,
         static_cast<T*>(k_out), static_cast<T*>(v_out), counts, ctx->ws.seg_start, ctx->ws.seg_end, ctx->ws.carry,
         ctx->ws.carry_cnt, n, cap, ctx->seg_chunks);
   }
@@ -530,7 +530,7 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
       {
         LaunchScope scope(ctx, MEDA_K_GROUP, st);
         sort_hist_kernel<<<grid, kSortWarps * 32, 0, st>>>(keys, budget_row, ctx->ws.sort_table, n, cap, shift,
-                                                           ctx->sort_chunks, ctx->ws.seg_start, ctx->ws.seg_end);
+                                                           ctx->sort_chunks);
       }
       {
         LaunchScope scope(ctx, MEDA_K_GROUP, st);
@@ -539,8 +539,9 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
       }
       {
         LaunchScope scope(ctx, MEDA_K_GROUP, st);
-        sort_scatter_kernel<<<grid, kSortWarps * 32, 0, st>>>(keys, rows, budget_row, ctx->ws.sort_table, ko, ro, n,
-                                                              cap, shift, ctx->sort_chunks);
+        sort_scatter_kernel<<<grid, kSortWarps * 32, 0, st>>>(keys, rows, idx_conserved, budget_row,
+                                                              ctx->ws.sort_table, ko, ro, n, cap, shift,
+                                                              ctx->sort_chunks);
       }
       keys = ko;
       rows = ro;

@@ -533,3 +533,42 @@ def test_pass_from_pinned_host_buffers_returns_what_the_device_pass_holds(wl):
         assert d2h == budgets.numel() * 4 + sum(t.numel() * t.element_size()
                                                 for name in ("k", "v", "counts", "idx") for t in out_host[name])
     cp.close()
+
+
+@pytest.mark.parametrize("wl", [
+    W.small_variant("capacity_2857", spans=W._spans((37, 0), (45 * 61, 1), (75, 0)), window=32, n_layers=6,
+                    rho=0.25, seed=15),
+    W.small_variant("capacity_f32", dtype="f32", n_q_heads=4, n_kv_heads=2, head_dim=128, n_layers=3, seed=16),
+], ids=lambda w: w.name)
+def test_output_capacity_smaller_than_the_prompt_gives_the_same_rows(wl):
+    """Outputs sized for the largest layer budget instead of the whole prompt (the stride of the kept-index
+    list and of the compacted caches changes in every phase-B kernel) hold the same bits in their live rows."""
+    from paper_2502_17599_b200.pipeline import CompressionPass
+    L, n = wl.n_layers, wl.n_tokens
+    qs, ks, vs = [], [], []
+    for l in range(L):
+        q, k, v = W.make_layer(wl, l, "cuda")
+        qs.append(q); ks.append(k); vs.append(v)
+    full = CompressionPass(wl)
+    full.run(qs, ks, vs)
+    full.check()
+    budgets = full.budgets.cpu().numpy()
+    s_max = int(budgets[:, 0].max())
+    assert s_max < n
+    assert budgets[:, 0].min() <= 384 or wl.dtype != "bf16"      # both arg-max kernels take part
+    tight = CompressionPass(wl, row_capacity=s_max)
+    tight.run(qs, ks, vs)
+    tight.check()
+    assert torch.equal(tight.budgets, full.budgets)
+    for l in range(L):
+        S = int(budgets[l, 0])
+        for a, b in ((tight.k_out, full.k_out), (tight.v_out, full.v_out), (tight.counts, full.counts),
+                     (tight.idx_c, full.idx_c)):
+            assert torch.equal(a[l][:, :S], b[l][:, :S]), l
+    # one row too few for the largest layer is reported, not written past
+    short = CompressionPass(wl, row_capacity=s_max - 1)
+    short.run(qs, ks, vs)
+    with pytest.raises(Exception):
+        short.check()
+    for c in (full, tight, short):
+        c.close()

@@ -337,16 +337,70 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
   end_piece(cur, started_here, ended, q1);
 }
 
-// One warp per (conserved slot, tensor): slots whose rows span several chunks get their parked pieces
-// added in chunk order (loaded eight at a time, added one by one); everything else was finished by the
-// walker.  Without merging (`evict`) the kept rows are copied.  grid = (blocks, heads, 2).
+// Finishes the slots whose rows span several chunks: one warp per (chunk border, tensor).  The slot that
+// crosses border b (the last row of chunk b - 1 and the first row of chunk b belong to it) is finished
+// by the warp of the FIRST border it crosses: the piece parked by the chunk where it starts, then the
+// pieces of the following chunks in chunk order (loaded eight at a time, added one by one), one division,
+// one rounding.  Everything else was finished by the walker.  grid = (blocks of 8 borders, heads, 2).
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
-seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ idx_conserved,
-                    const int32_t* __restrict__ budget_row, const int32_t* __restrict__ seg_start,
-                    const int32_t* __restrict__ seg_end, const float* __restrict__ carry,
-                    const int32_t* __restrict__ carry_cnt, T* __restrict__ k_out, T* __restrict__ v_out,
-                    int32_t* __restrict__ counts, int n, int cap, int n_chunks, int evict) {
+seg_border_kernel(const int32_t* __restrict__ keys_a, const int32_t* __restrict__ keys_b, int max_passes,
+                  const int32_t* __restrict__ budget_row, const int32_t* __restrict__ seg_start,
+                  const int32_t* __restrict__ seg_end, const float* __restrict__ carry,
+                  const int32_t* __restrict__ carry_cnt, T* __restrict__ k_out, T* __restrict__ v_out,
+                  int32_t* __restrict__ counts, int n, int cap, int n_chunks) {
+  constexpr int E = D / 32;
+  const int g = blockIdx.y, lane = threadIdx.x % 32;
+  const int tensor = blockIdx.z;
+  const int S = min(budget_row[0], cap);
+  const int border = blockIdx.x * 8 + threadIdx.x / 32 + 1;       // between chunks border - 1 and border
+  const int q = border * kSegChunk;
+  if (S <= 0 || q >= n) return;
+  const bool in_b = ((sort_passes_done(S, max_passes) - 1) & 1) != 0;
+  const int32_t* kg = (in_b ? keys_b : keys_a) + (size_t)g * n;
+  const int slot = min(max(kg[q - 1], 0), S - 1);
+  if (min(max(kg[q], 0), S - 1) != slot) return;                  // no slot crosses this border
+  const int start = seg_start[(size_t)g * n + slot], end = seg_end[(size_t)g * n + slot];
+  const int c0 = start / kSegChunk, c1 = (end - 1) / kSegChunk;
+  if (c0 != border - 1) return;                                   // an earlier border finishes this slot
+  T* out_g = (tensor == 0 ? k_out : v_out) + (size_t)g * cap * D;
+  float* base = const_cast<float*>(carry);
+  float acc[E];
+  const float* p = carry_ptr<D>(base, g, c0, 1, n_chunks) + tensor * D;
+#pragma unroll
+  for (int e = 0; e < E; ++e) acc[e] = p[lane * E + e];
+  int members = carry_cnt[((size_t)g * n_chunks + c0) * 2 + 1];
+  for (int cb = c0 + 1; cb <= c1; cb += 8) {
+    float x[8][E];
+    int m[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int c = min(cb + u, c1);
+      const float* pc = carry_ptr<D>(base, g, c, 0, n_chunks) + tensor * D;
+#pragma unroll
+      for (int e = 0; e < E; ++e) x[u][e] = pc[lane * E + e];
+      m[u] = carry_cnt[((size_t)g * n_chunks + c) * 2];
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (cb + u <= c1) {
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] += x[u][e];
+        members += m[u];
+      }
+    }
+  }
+  store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)members);
+  if (tensor == 0 && lane == 0) counts[(size_t)g * cap + slot] = members;
+}
+
+// Without merging (merge_mode 1) the kept rows are copied: one warp per (slot, tensor).
+// grid = (blocks, heads, 2).
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+copy_kept_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ idx_conserved,
+                 const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,
+                 int32_t* __restrict__ counts, int n, int cap) {
   constexpr int E = D / 32;
   const int g = blockIdx.y, lane = threadIdx.x % 32;
   const int tensor = blockIdx.z;
@@ -355,46 +409,11 @@ seg_finalize_kernel(const T* __restrict__ k, const T* __restrict__ v, const int3
   const int S = min(budget_row[0], cap);
   // the grid is sized on the host for the largest possible S: walk the slots with a stride
   for (int slot = blockIdx.x * 8 + threadIdx.x / 32; slot < S; slot += gridDim.x * 8) {
-    const int start = evict ? 0 : seg_start[(size_t)g * n + slot];
-    const int end = evict ? 0 : seg_end[(size_t)g * n + slot];
+    const int own = min(max(idx_conserved[(size_t)g * cap + slot], 0), n - 1);
     float acc[E];
-    int members = 0;
-    if (evict) {
-      const int own = min(max(idx_conserved[(size_t)g * cap + slot], 0), n - 1);
-      load_row<T, E>(x_g + (size_t)own * D, lane, acc);
-      members = 1;
-    } else {
-      if (end <= start) continue;                         // cannot happen: every slot has its kept row in the list
-      const int c0 = start / kSegChunk, c1 = (end - 1) / kSegChunk;
-      if (c0 == c1) continue;
-      float* base = const_cast<float*>(carry);
-      const float* p = carry_ptr<D>(base, g, c0, 1, n_chunks) + tensor * D;
-#pragma unroll
-      for (int e = 0; e < E; ++e) acc[e] = p[lane * E + e];
-      members = carry_cnt[((size_t)g * n_chunks + c0) * 2 + 1];
-      for (int cb = c0 + 1; cb <= c1; cb += 8) {
-        float x[8][E];
-        int m[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int c = min(cb + u, c1);
-          const float* pc = carry_ptr<D>(base, g, c, 0, n_chunks) + tensor * D;
-#pragma unroll
-          for (int e = 0; e < E; ++e) x[u][e] = pc[lane * E + e];
-          m[u] = carry_cnt[((size_t)g * n_chunks + c) * 2];
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (cb + u <= c1) {
-#pragma unroll
-            for (int e = 0; e < E; ++e) acc[e] += x[u][e];
-            members += m[u];
-          }
-        }
-      }
-    }
-    store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)members);
-    if (tensor == 0 && lane == 0) counts[(size_t)g * cap + slot] = members;
+    load_row<T, E>(x_g + (size_t)own * D, lane, acc);
+    store_row<T, E>(out_g + (size_t)slot * D, lane, acc, 1.f);
+    if (tensor == 0 && lane == 0) counts[(size_t)g * cap + slot] = 1;
   }
 }
 

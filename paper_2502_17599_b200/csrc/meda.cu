@@ -505,10 +505,16 @@ void launch_seg_kernels(meda_ctx* ctx, const void* k, const void* v, const int32
         ctx->ws.carry_cnt, n, cap, ctx->seg_chunks);
   }
   LaunchScope scope(ctx, MEDA_K_REDUCE, st);
-  seg_finalize_kernel<T, D><<<dim3(slot_blocks(ctx, max_slots, 8, 2 * c.n_kv_heads), c.n_kv_heads, 2), 256, 0, st>>>(
-      static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, budget_row, ctx->ws.seg_start,
-      ctx->ws.seg_end, ctx->ws.carry, ctx->ws.carry_cnt, static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n,
-      cap, ctx->seg_chunks, evict);
+  if (evict) {
+    copy_kept_kernel<T, D><<<dim3(slot_blocks(ctx, max_slots, 8, 2 * c.n_kv_heads), c.n_kv_heads, 2), 256, 0, st>>>(
+        static_cast<const T*>(k), static_cast<const T*>(v), idx_conserved, budget_row, static_cast<T*>(k_out),
+        static_cast<T*>(v_out), counts, n, cap);
+  } else {
+    seg_border_kernel<T, D><<<dim3((ctx->seg_chunks + 7) / 8, c.n_kv_heads, 2), 256, 0, st>>>(
+        ctx->ws.sort_keys[0], ctx->ws.sort_keys[1], ctx->sort_passes, budget_row, ctx->ws.seg_start, ctx->ws.seg_end,
+        ctx->ws.carry, ctx->ws.carry_cnt, static_cast<T*>(k_out), static_cast<T*>(v_out), counts, n, cap,
+        ctx->seg_chunks);
+  }
 }
 
 template <typename T>

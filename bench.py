@@ -36,7 +36,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long_video_128k")
     ap.add_argument("--layers", type=int, default=0, help="keep only the first N layers (profiling captures); 0 = all")
-    ap.add_argument("--streams", type=int, default=4, help="streams (and contexts) the layers alternate between")
+    ap.add_argument("--streams", type=int, default=8, help="streams (and contexts) the layers alternate between")
     ap.add_argument("--eager", action="store_true", help="time eager launches instead of a CUDA-graph replay of the pass")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")

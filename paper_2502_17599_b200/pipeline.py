@@ -17,7 +17,7 @@ class CompressionPass:
     `row_capacity` bounds S_l per layer (n_tokens is always safe; a smaller value saves memory and
     makes a layer whose budget exceeds it report MEDA_ERR_WORKSPACE)."""
 
-    def __init__(self, wl: Workload, row_capacity: int | None = None, device="cuda", n_streams: int = 4,
+    def __init__(self, wl: Workload, row_capacity: int | None = None, device="cuda", n_streams: int = 8,
                  **ctx_overrides):
         self.wl = wl
         self.device = device
@@ -66,7 +66,7 @@ class CompressionPass:
             main.wait_event(ev)
 
     def run(self, q_layers, k_layers, v_layers, stream=None, single_stream=False, qk_ready=None, v_ready=None,
-            budgets_done=None, layer_done=None):
+            budgets_done=None, layer_done=None, max_lanes=None):
         """Enqueues the whole pass.  Inputs are lists of per-layer device tensors; results stay on the
         device in this object's buffers.  The work is ordered after what `stream` (default: torch's
         current stream) holds and `stream` waits for all of it.  With `single_stream` everything goes to
@@ -75,13 +75,15 @@ class CompressionPass:
         place (copies still in flight on another stream): phase A of a layer waits for the first,
         phase B for the second.  `budgets_done` (an event) is recorded once the budgets are written,
         `layer_done[l]` (events) once layer l's compressed cache is: a caller can start copying results
-        out while later layers are still being compressed."""
+        out while later layers are still being compressed.  `max_lanes` limits the streams used."""
         L = self.wl.n_layers
         main = stream if stream is not None else torch.cuda.current_stream()
         if single_stream or not self.streams:
             lanes = [(self.contexts[0], main, self.row_stats[0])]
         else:
             lanes = list(zip(self.contexts, self.streams, self.row_stats))
+            if max_lanes is not None:
+                lanes = lanes[: max(1, max_lanes)]
             self._fork(main)
         for l in range(L):
             c, s, rs = lanes[l % len(lanes)]
@@ -158,7 +160,7 @@ class CompressionPass:
         budgets_done = torch.cuda.Event()
         layer_done = [torch.cuda.Event() for _ in range(L)]
         self.run(staging["q"], staging["k"], staging["v"], qk_ready=qk_ready, v_ready=v_ready,
-                 budgets_done=budgets_done, layer_done=layer_done)
+                 budgets_done=budgets_done, layer_done=layer_done, max_lanes=4)
         # Results leave on a third stream: the budgets as soon as they exist (the live row counts decide
         # what comes back), then each layer's compacted cache as soon as that layer is done, while the
         # values of later layers are still arriving (the link carries both directions at once).

@@ -213,8 +213,10 @@ def algorithmic_work(wl, budgets):
         small = split and s <= NEAREST_SMALL_MAX_S
         out["nearest_small_flops" if small else "nearest_flops"].append(2.0 * (n - s) * s * d * hkv if s < n else 0.0)
         out["reduce_bytes"].append(2 * hkv * n * d * e + 2 * hkv * s * d * e + 4 * hkv * s)
-        # grouping: every pass reads the (slot, row) pairs twice (histogram, scatter) and writes them once
-        out["group_bytes"].append(sort_passes * (8 + 4 + 8) * hkv * (n - s))
+        # grouping: all n rows are sorted by slot; a pass reads the (slot, row) pairs twice (histogram, scatter)
+        # and writes them once, and only the passes over digits that slots < S reach are executed
+        executed = min(sort_passes, 1 if s <= 512 else (2 if s <= 512 * 512 else 3))
+        out["group_bytes"].append(executed * (8 + 4 + 8) * hkv * n)
         out["select_bytes"].append(4 * hkv * n + 4 * hkv * n)
     return out
 

@@ -104,3 +104,26 @@ def test_tensor_core_kernels_keep_tensor_memory_loads_out_of_local_memory():
     assert len(hits) >= 6, "tensor-core kernels not found in the ptxas report"
     for i in hits:
         assert "0 bytes spill stores, 0 bytes spill loads" in lines[i + 1], (lines[i], lines[i + 1])
+
+
+def test_bench_work_accounting_matches_the_kernels_switch_points():
+    """bench.py splits the arg-max flops between the two kernels at the slot count the device code switches
+    at, and counts one grouping pass per 9-bit digit of the prompt length."""
+    import re
+    import bench
+    from paper_2502_17599_b200 import binding, workloads as W
+    src = open(os.path.join(ROOT, "paper_2502_17599_b200", "csrc", "nearest_sm100.cuh")).read()
+    assert int(re.search(r"kNearestSmallMaxS\s*=\s*(\d+)", src).group(1)) == binding.NEAREST_SMALL_MAX_S
+    wl = W.WORKLOADS["long_video_128k"]
+    n, d, hkv = wl.n_tokens, wl.head_dim, wl.n_kv_heads
+    budgets = [36, binding.NEAREST_SMALL_MAX_S, binding.NEAREST_SMALL_MAX_S + 1, 67970]
+    work = bench.algorithmic_work(wl, budgets)
+    flops = lambda s: 2.0 * (n - s) * s * d * hkv
+    assert work["nearest_small_flops"] == [flops(36), flops(binding.NEAREST_SMALL_MAX_S)]
+    assert work["nearest_flops"] == [flops(binding.NEAREST_SMALL_MAX_S + 1), flops(67970)]
+    assert work["group_bytes"][0] == 1 * 20 * hkv * n                 # 36 slots: one 9-bit digit, all n rows
+    assert work["group_bytes"][3] == 2 * 20 * hkv * n                 # 67,970 slots: two digits
+    assert all(b == hkv * n * d * 2 for b in work["stats_bytes"])
+    # fp32 workloads have no streaming kernel: everything is the generic kernel's
+    tiny = bench.algorithmic_work(W.WORKLOADS["tiny"], [100, 200])
+    assert tiny["nearest_small_flops"] == [] and len(tiny["nearest_flops"]) == 2

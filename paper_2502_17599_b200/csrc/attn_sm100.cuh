@@ -84,14 +84,10 @@ struct StatsPolicy {
       else z += fast_exp2(t - m);
     }
     // 32 consecutive keys starting at j0 against this thread's query row.
+    // uniform_text / uniform_visual: all 32 keys of the chunk are text / visual (the same for every row: the
+    // caller derives them once per tile from two warp votes).
     __device__ __forceinline__ void chunk(const Params& p, const uint32_t (&r)[32], int chunk_idx, int j0,
-                                          int last_visible) {
-      const uint4 ma = reinterpret_cast<const uint4*>(mod_t + chunk_idx * 32)[0];
-      const uint4 mb = reinterpret_cast<const uint4*>(mod_t + chunk_idx * 32)[1];
-      const uint32_t all_or = ma.x | ma.y | ma.z | ma.w | mb.x | mb.y | mb.z | mb.w;
-      const uint32_t all_and = ma.x & ma.y & ma.z & ma.w & mb.x & mb.y & mb.z & mb.w;
-      const bool uniform_text = all_or == 0u;
-      const bool uniform_visual = all_and == 0x01010101u && all_or == 0x01010101u;
+                                          int last_visible, bool uniform_text, bool uniform_visual) {
       if ((uniform_text || uniform_visual) && j0 + 31 <= last_visible) {
         // one modality, all keys visible: chunk maximum first (three-input maxima), then one exp2 per key
         float t[12];
@@ -135,8 +131,12 @@ struct StatsPolicy {
       const int last_visible = p.n - p.w + i;           // causal: keys j <= last_visible
       const int c0 = it.b_row + tile * 128;
       __syncwarp();
-      reinterpret_cast<uint32_t*>(mod_t)[lane] = __ldg(reinterpret_cast<const uint32_t*>(p.modality + c0) + lane);
+      const uint32_t mod4 = __ldg(reinterpret_cast<const uint32_t*>(p.modality + c0) + lane);   // keys 4 lane .. 4 lane + 3
+      reinterpret_cast<uint32_t*>(mod_t)[lane] = mod4;
       __syncwarp();
+      // which 32-key chunks hold one modality only: lanes 8 c .. 8 c + 7 cover chunk c
+      const uint32_t text4 = __ballot_sync(0xffffffffu, mod4 == 0u);
+      const uint32_t vis4 = __ballot_sync(0xffffffffu, mod4 == 0x01010101u);
       if (!__any_sync(0xffffffffu, valid)) return;
       // One chunk in registers at a time: with four epilogue warps per scheduler the load latency hides
       // behind the other warps, and a second buffer does not fit the 96 registers a 576-thread block
@@ -148,7 +148,9 @@ struct StatsPolicy {
         sm100::tmem_ld_32x32_issue(taddr + 32u * c, acc);
         sm100::tmem_ld_wait();
         sm100::tmem_ld_pin(acc);
-        if (valid) chunk(p, acc, c, c0 + 32 * c, last_visible);
+        if (valid)
+          chunk(p, acc, c, c0 + 32 * c, last_visible, ((text4 >> (8 * c)) & 0xffu) == 0xffu,
+                ((vis4 >> (8 * c)) & 0xffu) == 0xffu);
       }
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {

@@ -28,6 +28,27 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Packed fp32 pairs (sm_100): two fused multiply-adds / two additions per issue slot, each rounded exactly
+// like the scalar instruction.  Operands are pairs of fp32 in 64-bit registers.
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void f32x2_split(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Sweep 1: normalisers
 // ---------------------------------------------------------------------------------------------
@@ -102,14 +123,20 @@ struct StatsPolicy {
         float& m = uniform_visual ? mv : mt;
         float& z = uniform_visual ? zv : zt;
         const float m_new = fmaxf(m, cm * p.sc2);
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        // four running sums as two packed pairs: the scaling and the additions take half the issue slots
+        const uint64_t sc2x2 = f32x2(p.sc2, p.sc2), ref2 = f32x2(-m_new, -m_new);
+        uint64_t a01 = f32x2(0.f, 0.f), a23 = a01;
 #pragma unroll
         for (int x = 0; x < 32; x += 4) {
-          a0 += fast_exp2(fmaf(__uint_as_float(r[x + 0]), p.sc2, -m_new));
-          a1 += fast_exp2(fmaf(__uint_as_float(r[x + 1]), p.sc2, -m_new));
-          a2 += fast_exp2(fmaf(__uint_as_float(r[x + 2]), p.sc2, -m_new));
-          a3 += fast_exp2(fmaf(__uint_as_float(r[x + 3]), p.sc2, -m_new));
+          float t0, t1, t2, t3;
+          f32x2_split(fma_f32x2(sm100::pack_f32x2(r[x + 0], r[x + 1]), sc2x2, ref2), t0, t1);
+          f32x2_split(fma_f32x2(sm100::pack_f32x2(r[x + 2], r[x + 3]), sc2x2, ref2), t2, t3);
+          a01 = add_f32x2(a01, f32x2(fast_exp2(t0), fast_exp2(t1)));
+          a23 = add_f32x2(a23, f32x2(fast_exp2(t2), fast_exp2(t3)));
         }
+        float a0, a1, a2, a3;
+        f32x2_split(a01, a0, a1);
+        f32x2_split(a23, a2, a3);
         z = z * fast_exp2(m - m_new) + ((a0 + a1) + (a2 + a3));
         m = m_new;
       } else {

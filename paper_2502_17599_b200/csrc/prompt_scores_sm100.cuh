@@ -24,7 +24,7 @@
 namespace meda {
 
 constexpr float kPromptHidden = -1e30f;     // replaces a logit the causal mask hides: its exp2 is exactly 0
-constexpr float kPromptNoRow = 1e30f;       // reference of a row past the end of the prompt: every exp2 is 0
+constexpr float kPromptNoRow = -1e30f;      // negated reference of a row past the end of the prompt: every exp2 is 0
 
 // ---------------------------------------------------------------------------------------------
 // Pass 1: normalisers of every prompt row
@@ -86,14 +86,20 @@ struct PromptStatsPolicy {
         const float u2 = sm100::fmax3(t[6], t[7], t[8]), u3 = sm100::fmax3(t[9], t[10], t[11]);
         const float cm = fmaxf(sm100::fmax3(u0, u1, u2), u3);
         const float m_new = fmaxf(m, cm * p.sc2);
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        // four running sums as two packed pairs: the scaling and the additions take half the issue slots
+        const uint64_t sc2x2 = f32x2(p.sc2, p.sc2), ref2 = f32x2(-m_new, -m_new);
+        uint64_t a01 = f32x2(0.f, 0.f), a23 = a01;
 #pragma unroll
         for (int x = 0; x < 32; x += 4) {
-          a0 += fast_exp2(fmaf(__uint_as_float(acc[x + 0]), p.sc2, -m_new));
-          a1 += fast_exp2(fmaf(__uint_as_float(acc[x + 1]), p.sc2, -m_new));
-          a2 += fast_exp2(fmaf(__uint_as_float(acc[x + 2]), p.sc2, -m_new));
-          a3 += fast_exp2(fmaf(__uint_as_float(acc[x + 3]), p.sc2, -m_new));
+          float t0, t1, t2, t3;
+          f32x2_split(fma_f32x2(sm100::pack_f32x2(acc[x + 0], acc[x + 1]), sc2x2, ref2), t0, t1);
+          f32x2_split(fma_f32x2(sm100::pack_f32x2(acc[x + 2], acc[x + 3]), sc2x2, ref2), t2, t3);
+          a01 = add_f32x2(a01, f32x2(fast_exp2(t0), fast_exp2(t1)));
+          a23 = add_f32x2(a23, f32x2(fast_exp2(t2), fast_exp2(t3)));
         }
+        float a0, a1, a2, a3;
+        f32x2_split(a01, a0, a1);
+        f32x2_split(a23, a2, a3);
         z = z * fast_exp2(m - m_new) + ((a0 + a1) + (a2 + a3));
         m = m_new;
       } else {
@@ -132,8 +138,8 @@ struct PromptStatsPolicy {
   };
 };
 
-// ref[h][r] = max + log2(sum) of row r over both partials (base-2 units); rows past the end of the prompt
-// (the padding up to n_pad) get a reference no logit reaches.
+// ref[h][r] = -(max + log2(sum)) of row r over both partials (base-2 units, negated: the sweep adds it);
+// rows past the end of the prompt (the padding up to n_pad) get a reference no logit reaches.
 __global__ void __launch_bounds__(256)
 prompt_ref_kernel(const float2* __restrict__ partial, float* __restrict__ ref, int hq, int n, int n_pad) {
   const size_t total = (size_t)hq * n_pad;
@@ -144,7 +150,7 @@ prompt_ref_kernel(const float2* __restrict__ partial, float* __restrict__ ref, i
       const float2 a = partial[e], b = partial[total + e];
       const float m = fmaxf(a.x, b.x);                  // finite: every row sees itself
       const float z = a.y * fast_exp2(a.x - m) + b.y * fast_exp2(b.x - m);
-      out = m + log2f(z);
+      out = -(m + log2f(z));
     }
     ref[e] = out;
   }
@@ -164,7 +170,7 @@ __host__ __device__ inline int prompt_block_splits(int n, int blk, int splits) {
 
 struct PromptSweepPolicy {
   struct Params {
-    const float* ref;            // [Hq][n_pad]
+    const float* ref;            // [Hq][n_pad], negated references
     float* partial;              // [splits * 2][Hkv][n]: one slot per (row run, epilogue group)
     int n, n_pad, hq, hkv, group;
     int n_blocks;                // ceil(n / 256)
@@ -216,7 +222,7 @@ struct PromptSweepPolicy {
   struct Epilogue {
     int lane, row_in_block, egroup;
     float score;                 // this thread's key, summed over the tiles and heads of the unit so far
-    float s0, s1, s2, s3;        // partial sums inside one tile: small addends meet a small running sum
+    uint64_t s01, s23;           // partial sums inside one tile (packed pairs): small addends meet a small running sum
     __device__ void init(const Params&, unsigned char*, int ewarp, int lane_) {
       lane = lane_;
       egroup = ewarp / kUsEpilogueWarps;
@@ -231,13 +237,16 @@ struct PromptSweepPolicy {
 #pragma unroll
         for (int x = 0; x < 32; ++x) if (r0 + x < j) acc[x] = __float_as_uint(kPromptHidden);
       }
+      const uint64_t sc2x2 = f32x2(p.sc2, p.sc2);
 #pragma unroll
       for (int x = 0; x < 32; x += 4) {
-        const float4 c = __ldg(ref4 + x / 4);             // references of rows r0 + x .. r0 + x + 3
-        s0 += fast_exp2(fmaf(__uint_as_float(acc[x + 0]), p.sc2, -c.x));
-        s1 += fast_exp2(fmaf(__uint_as_float(acc[x + 1]), p.sc2, -c.y));
-        s2 += fast_exp2(fmaf(__uint_as_float(acc[x + 2]), p.sc2, -c.z));
-        s3 += fast_exp2(fmaf(__uint_as_float(acc[x + 3]), p.sc2, -c.w));
+        // negated references of rows r0 + x .. r0 + x + 3, as two packed pairs
+        const ulonglong2 c = __ldg(reinterpret_cast<const ulonglong2*>(ref4) + x / 4);
+        float t0, t1, t2, t3;
+        f32x2_split(fma_f32x2(sm100::pack_f32x2(acc[x + 0], acc[x + 1]), sc2x2, c.x), t0, t1);
+        f32x2_split(fma_f32x2(sm100::pack_f32x2(acc[x + 2], acc[x + 3]), sc2x2, c.y), t2, t3);
+        s01 = add_f32x2(s01, f32x2(fast_exp2(t0), fast_exp2(t1)));
+        s23 = add_f32x2(s23, f32x2(fast_exp2(t2), fast_exp2(t3)));
       }
     }
     __device__ void tile(const Params& p, const StreamItem& it, int tile, uint32_t taddr) {
@@ -246,7 +255,7 @@ struct PromptSweepPolicy {
       const int warp_first = j - lane;                  // the warp's first key is seen by the most rows
       const int r_tile = it.b_row + tile * 128;
       const float4* ref4 = reinterpret_cast<const float4*>(p.ref + (size_t)it.u0 * p.n_pad + r_tile);
-      s0 = s1 = s2 = s3 = 0.f;
+      s01 = s23 = f32x2(0.f, 0.f);
       // one chunk in registers at a time (sixteen epilogue warps hide the load latency for each other, and
       // a block of this size has no registers for a second buffer)
       uint32_t acc[32];
@@ -258,6 +267,9 @@ struct PromptSweepPolicy {
         sm100::tmem_ld_pin(acc);
         if (valid) chunk(p, acc, ref4 + 8 * c, r_tile + 32 * c, j);
       }
+      float s0, s1, s2, s3;
+      f32x2_split(s01, s0, s1);
+      f32x2_split(s23, s2, s3);
       score += (s0 + s1) + (s2 + s3);
     }
     __device__ void item_end(const Params& p, const StreamItem& it) {

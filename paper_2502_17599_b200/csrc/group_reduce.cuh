@@ -242,7 +242,7 @@ __device__ __forceinline__ void store_row(T* p, int lane, const float (&x)[E], f
 // as many warps keep rows in flight; the z = 0 warps also record segment bounds and counts.  Every slot
 // has at least one row in the list (its kept row), so every slot's bounds get written.
 template <typename T, int D>
-__global__ void __launch_bounds__(kSegWarps * 32, 9)
+__global__ void __launch_bounds__(kSegWarps * 32, 10)
 seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* __restrict__ keys_a,
                   const int32_t* __restrict__ rows_a, const int32_t* __restrict__ keys_b,
                   const int32_t* __restrict__ rows_b, int max_passes, const int32_t* __restrict__ budget_row, T* __restrict__ k_out, T* __restrict__ v_out,

@@ -271,6 +271,11 @@ const char* meda_kernel_class_name(int32_t kernel_class);
  * still counted but no longer timed. */
 meda_status meda_profile_enable(meda_ctx* ctx, int32_t enable);
 
+/* Launches since the last meda_profile_read (or meda_profile_enable) that were NOT timed because
+ * the event pool was full.  Per-class times of such a record cover only part of the launches:
+ * a caller that divides them by a step count must check that this is 0. */
+int64_t meda_profile_dropped(const meda_ctx* ctx);
+
 /* Synchronises the recorded events and writes, per kernel class, the summed device time in
  * milliseconds (ms_out, HOST float[MEDA_K_CLASSES]) and the number of timed launches
  * (launches_out, HOST int32[MEDA_K_CLASSES]); then clears the record.  Either pointer may be NULL. */
@@ -278,6 +283,15 @@ meda_status meda_profile_read(meda_ctx* ctx, float* ms_out, int32_t* launches_ou
 
 /* Number of kernels this context has launched since it was created (timing on or off). */
 int64_t meda_launch_count(const meda_ctx* ctx);
+
+/* Self-test of the failure path every tensor-core pipeline of the library shares (no counterpart in
+ * the paper).  Each device-side wait of those pipelines is bounded: when it runs out, the kernel
+ * records MEDA_ERR_TIMEOUT in the context's status word, releases what it holds and returns.  This
+ * call launches one small block that waits, with that same routine, on a barrier nothing arrives
+ * on, for at most `wait_cycles` cycles of the SM clock (1 .. 2e9; a few thousand is enough), so the
+ * path can be exercised without breaking a real kernel: afterwards meda_poll_status returns
+ * MEDA_ERR_TIMEOUT once, and the context works as before.  Nothing else is touched. */
+meda_status meda_selftest_wait_timeout(meda_ctx* ctx, int64_t wait_cycles, void* stream);
 
 #ifdef __cplusplus
 }

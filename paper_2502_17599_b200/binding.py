@@ -65,6 +65,8 @@ EXPORTS = {
     "meda_profile_enable": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
     "meda_profile_read": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]),
     "meda_launch_count": (ctypes.c_int64, [ctypes.c_void_p]),
+    "meda_profile_dropped": (ctypes.c_int64, [ctypes.c_void_p]),
+    "meda_selftest_wait_timeout": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]),
     "meda_window_scores": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
     "meda_window_scores_from_stats": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 6),
     "meda_prompt_scores_scratch_bytes": (ctypes.c_int64, [ctypes.c_void_p]),
@@ -197,6 +199,14 @@ class Context:
         cnt = (ctypes.c_int32 * n)()
         _check(self._lib.meda_profile_read(self._h, ms, cnt), "meda_profile_read")
         return {self._lib.meda_kernel_class_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
+
+    def profile_dropped(self) -> int:
+        """Launches since the last profile_read that went untimed because the event pool was full."""
+        return int(self._lib.meda_profile_dropped(self._h))
+
+    def selftest_wait_timeout(self, wait_cycles: int = 20000, stream=None):
+        _check(self._lib.meda_selftest_wait_timeout(self._h, int(wait_cycles), _stream(stream)),
+               "meda_selftest_wait_timeout")
 
     def poll_status(self, stream=None) -> int:
         return int(self._lib.meda_poll_status(self._h, _stream(stream)))

@@ -110,6 +110,8 @@ struct LaunchScope {
       slot = p.used++;
       p.klass[slot] = klass;
       cudaEventRecord(p.begin[slot], st);
+    } else if (p.enabled) {
+      ++p.dropped;
     }
   }
   ~LaunchScope() {
@@ -920,9 +922,12 @@ meda_status meda_profile_enable(meda_ctx* ctx, int32_t enable) {
     }
   }
   p.used = 0;
+  p.dropped = 0;
   p.enabled = true;
   return MEDA_OK;
 }
+
+int64_t meda_profile_dropped(const meda_ctx* ctx) { return ctx ? ctx->prof.dropped : 0; }
 
 meda_status meda_profile_read(meda_ctx* ctx, float* ms_out, int32_t* launches_out) {
   if (!ctx) return MEDA_ERR_INVALID_ARG;
@@ -937,6 +942,7 @@ meda_status meda_profile_read(meda_ctx* ctx, float* ms_out, int32_t* launches_ou
     cnt[p.klass[i]] += 1;
   }
   p.used = 0;
+  p.dropped = 0;
   if (ms_out) memcpy(ms_out, ms, sizeof(ms));
   if (launches_out) memcpy(launches_out, cnt, sizeof(cnt));
   return MEDA_OK;
@@ -949,6 +955,12 @@ meda_status meda_poll_status(meda_ctx* ctx, void* stream) {
   MEDA_CUDA_TRY(cudaMemcpy(&code, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost));
   if (code != 0) MEDA_CUDA_TRY(cudaMemset(ctx->ws.status, 0, sizeof(int)));
   return (meda_status)code;
+}
+
+meda_status meda_selftest_wait_timeout(meda_ctx* ctx, int64_t wait_cycles, void* stream) {
+  if (!ctx || wait_cycles < 1 || wait_cycles > 2000000000ll) return MEDA_ERR_INVALID_ARG;
+  wait_timeout_selftest_kernel<<<1, 64, 0, as_stream(stream)>>>((long long)wait_cycles, ctx->ws.status);
+  return launch_status();
 }
 
 meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, float* row_stats,

@@ -50,6 +50,7 @@ struct Profiler {
   cudaEvent_t* end = nullptr;     // [kPool]
   int* klass = nullptr;           // [kPool]
   int used = 0;
+  int64_t dropped = 0;            // launches since the last read that found the pool full and went untimed
 };
 }  // namespace meda
 

@@ -240,4 +240,25 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   if (threadIdx.x == 0 && *abort_flag != 0) set_status(status, MEDA_ERR_TIMEOUT);
 }
 
+// Exercises the give-up path of the bounded waits on its own: one block waits on a barrier that
+// nothing ever arrives on, with the given cycle limit.  The wait returns false, the block records
+// MEDA_ERR_TIMEOUT exactly like the pipelines above do on their exit path, and returns; nothing is
+// left waiting and no product kernel is involved.
+__global__ void wait_timeout_selftest_kernel(long long limit_cycles, int* status) {
+  using namespace sm100;
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  // every thread waits, as the roles of a pipeline would: the first to run out raises the flag,
+  // the others see it and leave too
+  const bool ok = mbar_wait(&bar, 0u, &abort_flag, limit_cycles);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || abort_flag != 0)) set_status(status, MEDA_ERR_TIMEOUT);
+}
+
 }  // namespace meda

@@ -1,11 +1,15 @@
 """GPU parity at the full benchmark sizes, in the launch configuration bench.py times (the
 CompressionPass sequence: window_scores per layer, allocate_budgets, compress_layer per layer).
 
-The oracle cannot run a whole 129K-token pass in test time, so what it can compute one by one is
-sampled: budgets of all layers (bit-exact), the entropy and the per-key scores of one layer, the
-selection of two heads, the arg-max target of a few hundred less-important rows and the merged rows
-of a few dozen slots; properties that hold at any size (every token accounted for, ascending
-indices, the recent window kept) are checked in full."""
+Phase A costs the oracle a window-by-prompt product per head, so EVERY layer's entropy, per-key
+scores and row normalisers are compared with it.  Phase B is checked in full where the oracle can
+afford it: the selection of every KV head of four layers (largest, smallest and two middle budgets),
+and, for one head of the layer with the largest budget and of a layer on the small-budget arg-max
+kernel, every arg-max target (the oracle's similarity evaluated block by block) and every merged
+slot.  Properties that hold at any size (every token accounted for, ascending indices, the recent
+window kept, bit-identical reruns) are checked for all layers and heads."""
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 import torch
@@ -23,8 +27,34 @@ def _built():
     build.build()
 
 
+def _oracle_phase_a(q, k, mod):
+    """(entropy, scores, row_stats) of one layer from the oracle, on the bits the device saw."""
+    qh, kh = P.np64(q), P.np64(k)
+    return O.cross_modal_entropy(qh, kh, mod), O.window_scores(qh, kh), O.row_stats(qh, kh, mod)
+
+
+def _detail_layers(budgets, n, small_max):
+    """Layers whose phase B is compared in detail: the largest budget that still merges something, the
+    smallest, two in between, and (when there is one) the largest budget that the small-budget arg-max
+    kernel serves."""
+    S = budgets[:, 0]
+    merging = [int(l) for l in np.argsort(-S, kind="stable") if S[l] < n]
+    picks = [merging[0], merging[-1], merging[len(merging) // 3], merging[(2 * len(merging)) // 3]]
+    small = [l for l in merging if S[l] <= small_max]
+    large = [l for l in merging if S[l] > small_max]
+    full = [merging[0]]
+    if small:
+        picks.append(small[0])
+        full.append(small[0])
+    if large and large[-1] not in full:
+        full.append(large[-1])                     # the smallest budget on the row-gathering kernel
+        picks.append(large[-1])
+    return sorted(set(picks)), full
+
+
 @pytest.mark.parametrize("name", ["multi_image_8k", "long_video_19k", "multimodal_32k", "long_video_128k"])
-def test_full_size_pass_sampled_against_the_oracle(name):
+def test_full_size_pass_against_the_oracle(name, parity_report):
+    from paper_2502_17599_b200.binding import NEAREST_SMALL_MAX_S
     from paper_2502_17599_b200.pipeline import CompressionPass
     wl = W.WORKLOADS[name]
     n, L, hkv, d = wl.n_tokens, wl.n_layers, wl.n_kv_heads, wl.head_dim
@@ -50,8 +80,25 @@ def test_full_size_pass_sampled_against_the_oracle(name):
         assert torch.equal(a, b_)
     del first, first_live
 
-    # ---- budgets: bit-exact from the entropies the device produced; they sum to the global budget
+    # ---- phase A of EVERY layer against the oracle: entropy, per-key scores, row normalisers
     ent = P.np64(cp.entropy)
+    buf = P.GpuBuffers(wl)
+    a_or = {}
+    with ThreadPoolExecutor(max_workers=4) as pool:
+        jobs = [pool.submit(_oracle_phase_a, qs[l], ks[l], mod) for l in range(L)]
+        for l in range(L):
+            # the same call outside the pass, to see the layer's normalisers: same kernels, same bits
+            cp.ctx.window_scores(l, qs[l], ks[l], buf.row_stats, buf.scores, buf.entropy)
+            cp.ctx.check()
+            assert torch.equal(buf.scores, cp.scores[l]) and float(buf.entropy[l]) == float(cp.entropy[l])
+            want_e, want_a, want_rs = jobs[l].result()
+            jobs[l] = None
+            P.assert_entropy_close(ent[l], want_e)
+            P.assert_scores_close(P.np64(cp.scores[l]), want_a)
+            P.assert_row_stats_close(P.np64(buf.row_stats), want_rs)
+            a_or[l] = want_a
+
+    # ---- budgets: bit-exact from the entropies the device produced; they sum to the global budget
     budgets = cp.budgets.cpu().numpy()
     np.testing.assert_array_equal(budgets, O.allocate_budgets(ent, wl.global_budget, n, wl.min_budget))
     assert int(budgets[:, 0].sum()) == wl.global_budget
@@ -68,61 +115,41 @@ def test_full_size_pass_sampled_against_the_oracle(name):
         sc = cp.scores[l].sum(dim=1).cpu().numpy()
         np.testing.assert_allclose(sc, (wl.n_q_heads // hkv) * wl.window, rtol=2e-4)
 
-    # ---- one layer in detail: the one with the largest budget that still merges something
-    order = np.argsort(-budgets[:, 0])
-    layer = int(next(l for l in order if budgets[l, 0] < n))
-    S, M, N = (int(x) for x in budgets[layer])
-    qh = P.np64(qs[layer])
-    kh = np.stack([P.np64(ks[layer][g]) for g in range(hkv)])
-    P.assert_entropy_close(ent[layer], O.cross_modal_entropy(qh, kh, mod))
-    a_or = O.window_scores(qh, kh)
-    a_gpu = P.np64(cp.scores[layer])
-    P.assert_scores_close(a_gpu, a_or)
-
-    # the same layer through the separate entry points, to see the targets; same kernels, same bits
-    buf = P.GpuBuffers(wl)
-    cp.ctx.select_topk(layer, cp.scores[layer], cp.budgets, buf.idx_c, buf.idx_less, buf.cap)
-    cp.ctx.merge_kv(layer, ks[layer], vs[layer], cp.budgets, buf.idx_c, buf.idx_less, buf.k_out, buf.v_out,
-                    buf.counts, buf.target, buf.cap)
-    cp.ctx.check()
-    assert torch.equal(buf.idx_c[:, :S], cp.idx_c[layer, :, :S])
-    assert torch.equal(buf.k_out[:, :S], cp.k_out[layer, :, :S]) and torch.equal(buf.v_out[:, :S], cp.v_out[layer, :, :S])
-    assert torch.equal(buf.counts[:, :S], cp.counts[layer, :, :S])
-
-    rng = np.random.default_rng(3)
-    swaps = ties = 0
-    for g in sorted({0, hkv - 1}):
+    # ---- phase B in detail
+    detail, full = _detail_layers(budgets, n, NEAREST_SMALL_MAX_S if (wl.dtype == "bf16" and d == 128) else 0)
+    swaps = ties = ulp_used = 0
+    checked_rows = checked_slots = 0
+    for layer in detail:
+        S, M, N = (int(x) for x in budgets[layer])
+        # the layer through the separate entry points, to see the less-important list and the targets
+        cp.ctx.select_topk(layer, cp.scores[layer], cp.budgets, buf.idx_c, buf.idx_less, buf.cap)
+        cp.ctx.merge_kv(layer, ks[layer], vs[layer], cp.budgets, buf.idx_c, buf.idx_less, buf.k_out, buf.v_out,
+                        buf.counts, buf.target, buf.cap)
+        cp.ctx.check()
+        assert torch.equal(buf.idx_c[:, :S], cp.idx_c[layer, :, :S])
+        assert torch.equal(buf.k_out[:, :S], cp.k_out[layer, :, :S]) and torch.equal(buf.v_out[:, :S], cp.v_out[layer, :, :S])
+        assert torch.equal(buf.counts[:, :S], cp.counts[layer, :, :S])
+        for g in range(hkv):                       # selection of every KV head against the oracle's scores
+            cons = buf.idx_c[g, :S].cpu().numpy().astype(np.int64)
+            less = buf.idx_less[g, : n - S].cpu().numpy().astype(np.int64)
+            swaps += P.compare_selection(cons, a_or[layer][g], mod, M, N)
+            np.testing.assert_array_equal(less, np.setdiff1d(np.arange(n), cons))
+        if layer not in full or S >= n:
+            continue
+        g = (layer * 7 + 1) % hkv                  # one head per layer, not always the first
+        kh, vh = P.np64(ks[layer][g]), P.np64(vs[layer][g])
         cons = buf.idx_c[g, :S].cpu().numpy().astype(np.int64)
         less = buf.idx_less[g, : n - S].cpu().numpy().astype(np.int64)
-        swaps += P.compare_selection(cons, a_or[g], mod, M, N)
-        np.testing.assert_array_equal(less, np.setdiff1d(np.arange(n), cons))
         tgt = buf.target[g, : n - S].cpu().numpy().astype(np.int64)
-        assert tgt.min() >= 0 and tgt.max() < S
-        # sampled arg-max targets
-        pick = rng.choice(n - S, size=min(256, n - S), replace=False)
-        u = O.cosine_similarity(kh[g][less[pick]], kh[g][cons])
-        want = np.argmax(u, axis=1)
-        diff = np.nonzero(want != tgt[pick])[0]
-        if diff.size:
-            gap = u[diff, want[diff]] - u[diff, tgt[pick][diff]]
-            assert (gap <= P.TARGET_ATOL).all(), float(gap.max())
-        ties += int(diff.size)
-        # sampled merged slots: the oracle's average over the members the device assigned
-        vh = P.np64(vs[layer][g])
-        slots = np.unique(np.concatenate([rng.choice(S, size=min(48, S), replace=False), tgt[pick[:16]]]))
-        got_k = P.np64(buf.k_out[g, :S])
-        got_v = P.np64(buf.v_out[g, :S])
-        cnt = buf.counts[g, :S].cpu().numpy()
-        for s in slots:
-            members = less[tgt == s]
-            rows = np.concatenate([[cons[s]], members])
-            assert cnt[s] == rows.size
-            for got, src in ((got_k[s], kh[g]), (got_v[s], vh)):
-                want_row = O.round_to_dtype(src[rows].sum(axis=0) / rows.size, wl.dtype)
-                err = np.abs(got - want_row)
-                ulp = np.where(np.abs(want_row) >= 8.0, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want_row), 1e-30))) - 7), 0.0)
-                assert ((err <= P.MERGE_BF16_ATOL) | (err <= ulp)).all(), (int(s), float(err.max()))
-    print(f"{name}: layer {layer} (S={S}): tolerated selection swaps {swaps}, sampled arg-max near-ties {ties}")
+        ties += P.compare_targets_blockwise(tgt, kh, cons, less)                # every less-important row
+        st = P.compare_merged(P.np64(buf.k_out[g, :S]), P.np64(buf.v_out[g, :S]), buf.counts[g, :S].cpu().numpy(),
+                              kh, vh, cons, less, tgt, wl.dtype)                # every merged slot
+        ulp_used += st["ulp_allowance_used"]
+        checked_rows += less.size
+        checked_slots += S
+    parity_report(f"{name}: phase A of all {L} layers in tolerance; selection of all {hkv} heads of layers {detail}: "
+                  f"{swaps} tolerated swaps; layers {full} (one head each): {checked_rows} arg-max rows with {ties} "
+                  f"tolerated near-ties, {checked_slots} merged slots with {ulp_used} elements on the one-ulp allowance")
     cp.close()
 
 

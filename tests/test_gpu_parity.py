@@ -200,7 +200,7 @@ def test_select_reports_capacity_and_bad_budget_rows():
 
 @pytest.mark.parametrize("wl", small_cases(), ids=lambda w: w.name)
 @pytest.mark.parametrize("merge_mode", [0, 1])
-def test_merge_kv_against_oracle_sets(wl, merge_mode):
+def test_merge_kv_against_oracle_sets(wl, merge_mode, parity_report):
     ctx = make_ctx(wl, merge_mode=merge_mode)
     buf = P.GpuBuffers(wl)
     mod = wl.modality().numpy()
@@ -225,7 +225,7 @@ def test_merge_kv_against_oracle_sets(wl, merge_mode):
             P.compare_merged(P.np64(buf.k_out[g, :S]), P.np64(buf.v_out[g, :S]), buf.counts[g, :S].cpu().numpy(),
                              kh[g], vh[g], c, ls, tgt, wl.dtype, merge_mode)
             assert (buf.k_out[g, S:] == 7.0).all()       # rows past S_l are left untouched
-    print(f"{wl.name}: tolerated arg-max near-ties: {near_ties}")
+    parity_report(f"merge_kv on the oracle's sets, {wl.name}, merge_mode {merge_mode}: tolerated arg-max near-ties {near_ties}")
     ctx.close()
 
 
@@ -306,7 +306,7 @@ def reseeded_cases():
 
 
 @pytest.mark.parametrize("wl", small_cases() + reseeded_cases(), ids=lambda w: w.name)
-def test_end_to_end_with_teacher_forcing(wl):
+def test_end_to_end_with_teacher_forcing(wl, parity_report):
     ctx = make_ctx(wl)
     buf = P.GpuBuffers(wl)
     mod = wl.modality().numpy()
@@ -327,7 +327,7 @@ def test_end_to_end_with_teacher_forcing(wl):
     budgets = buf.budgets.cpu().numpy()
     np.testing.assert_array_equal(budgets, O.allocate_budgets(ent, wl.global_budget, n, wl.min_budget))
     raw = O.allocate_budgets(np.array([O.cross_modal_entropy(h[0], h[1], mod) for h in host]), wl.global_budget, n, wl.min_budget)
-    print(f"{wl.name}: budgets differing from the un-forced oracle: {int((raw != budgets).any(axis=1).sum())} of {wl.n_layers}")
+    unforced = int((raw != budgets).any(axis=1).sum())
     swaps = ties = 0
     buf2 = P.GpuBuffers(wl)
     for l in range(wl.n_layers):
@@ -354,7 +354,8 @@ def test_end_to_end_with_teacher_forcing(wl):
             ties += P.compare_targets(tgt, host[l][1][g], cons, less)
             P.compare_merged(P.np64(buf.k_out[g, :S]), P.np64(buf.v_out[g, :S]), buf.counts[g, :S].cpu().numpy(),
                              host[l][1][g], host[l][2][g], cons, less, tgt, wl.dtype)
-    print(f"{wl.name}: tolerated selection swaps {swaps}, tolerated arg-max near-ties {ties}")
+    parity_report(f"end to end, {wl.name}: budget rows differing from the un-forced oracle {unforced} of {wl.n_layers}, "
+                  f"tolerated selection swaps {swaps}, tolerated arg-max near-ties {ties}")
     ctx.close()
 
 

@@ -406,6 +406,58 @@ def test_compress_pass_accounts_for_every_token():
     assert (np.diff(res["budgets"][order, 0]) >= 0).all()
 
 
+def test_compress_pass_is_the_composition_of_its_pinned_steps():
+    """The whole pass and the per-layer wrapper against the individually pinned steps called by hand,
+    on a prompt whose recent and important shares differ (M != N), so that handing the two sizes over
+    in the wrong order, taking the scores of another layer or head, or merging with another head's
+    keys cannot pass.  The split itself is checked from its definition: the last M_l tokens are all
+    kept, exactly N_l earlier ones are, and those are text tokens first, then the best-scored."""
+    from paper_2502_17599_b200 import workloads as W
+    wl = W.small_variant(name="pin_compose", seed=21, rho=0.3)
+    n, hkv = wl.n_tokens, wl.n_kv_heads
+    layers = [tuple(t.to(torch.float64).numpy() for t in W.make_layer(wl, l)) for l in range(wl.n_layers)]
+    mod = wl.modality().numpy()
+    res = O.compress_pass(layers, mod, wl.global_budget, wl.min_budget, wl.dtype, beta_recent=3, beta_important=1)
+    ent = np.array([O.cross_modal_entropy(q, k, mod) for q, k, _ in layers])
+    np.testing.assert_array_equal(res["entropy"], ent)
+    budgets = O.allocate_budgets(ent, wl.global_budget, n, wl.min_budget, 3, 1)
+    np.testing.assert_array_equal(res["budgets"], budgets)
+    assert (budgets[:, 1] != budgets[:, 2]).all()                      # M_l != N_l: the order of the two matters
+    n_text_early = [int((mod[: n - int(m)] == O.TEXT).sum()) for m in budgets[:, 1]]
+    for l, (q, k, v) in enumerate(layers):
+        S, M, N = (int(x) for x in budgets[l])
+        a_s = O.window_scores(q, k)
+        np.testing.assert_array_equal(res["scores"][l], a_s)
+        for g in range(hkv):
+            r = res["layers"][l][g]
+            cons, less = O.select_topk(a_s[g], mod, M, N)                # (recent, important) in this order
+            np.testing.assert_array_equal(r["conserved"], cons)
+            np.testing.assert_array_equal(r["less"], less)
+            # the split from its definition (Eq. 10), without select_topk
+            kept = np.zeros(n, dtype=bool)
+            kept[r["conserved"]] = True
+            assert kept[n - M:].all() and int(kept[: n - M].sum()) == N
+            early_text = np.nonzero((mod[: n - M] == O.TEXT))[0]
+            if N >= n_text_early[l]:
+                assert kept[early_text].all()                            # Eq. 9: text outranks every visual token
+            else:
+                assert not kept[: n - M][mod[: n - M] == O.VISUAL].any()
+            # merging with this head's keys and values, and the output rounding
+            km, vm, counts, target = O.merge_kv(k[g], v[g], cons, less)
+            np.testing.assert_array_equal(r["target"], target)
+            np.testing.assert_array_equal(r["counts"], counts)
+            np.testing.assert_array_equal(r["k"], O.round_to_dtype(km, wl.dtype))
+            np.testing.assert_array_equal(r["v"], O.round_to_dtype(vm, wl.dtype))
+        # the per-layer wrapper alone, same arguments in the same order
+        alone = O.compress_layer(k, v, a_s, mod, M, N, wl.dtype)
+        for g in range(hkv):
+            for key in ("conserved", "less", "target", "k", "v", "counts"):
+                np.testing.assert_array_equal(alone[g][key], res["layers"][l][g][key])
+    # heads of one layer and layers of one prompt really differ (a mix-up would show)
+    assert not np.array_equal(res["layers"][0][0]["conserved"], res["layers"][0][1]["conserved"])
+    assert not np.array_equal(res["layers"][0][0]["k"][:8], res["layers"][1][0]["k"][:8])
+
+
 def test_table6_headlines_and_memory_formula():
     rows, head = [], None
     with open(os.path.join(os.path.dirname(__file__), "golden", "table6_kv_memory.txt")) as f:

@@ -20,6 +20,7 @@
 #include "nearest_small_sm100.cuh"
 #include "prompt_scores_sm100.cuh"
 #include "select.cuh"
+#include "window_stats_sm100.cuh"
 
 using namespace meda;
 
@@ -59,6 +60,8 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.kc);
   cudaFree(ws.coef_vis);
   cudaFree(ws.coef_text);
+  cudaFree(ws.tile_class);
+  cudaFree(ws.stats_counters);
   for (int i = 0; i < 2; ++i) { cudaFree(ws.sort_keys[i]); cudaFree(ws.sort_rows[i]); }
   cudaFree(ws.sort_table);
   cudaFree(ws.seg_start);
@@ -205,17 +208,23 @@ meda_status launch_sweep(meda_ctx* ctx, int32_t layer, const void* q_win, const 
   return launch_status();
 }
 
-// bf16, head_dim 128, window 32 or 64: both sweeps on the tensor cores.
+// bf16, head_dim 128, window 32 or 64: both sweeps on the tensor cores.  The normaliser sweep also merges its
+// partial results (the last warp to finish a set of rows does) and writes the per-column constants of the
+// second sweep, so no other launch is needed in between.
 meda_status launch_stats_fast(meda_ctx* ctx, const void* q_win, const void* k, float* row_stats, cudaStream_t st) {
   const meda_config& c = ctx->cfg;
   if (((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(q_win)) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
-  CUtensorMap map_q, map_k;
-  if (!make_rows_map(ctx, &map_q, q_win, (int64_t)c.n_q_heads * c.window, 1, (int64_t)c.n_q_heads * c.window, 128) ||
-      !make_rows_map(ctx, &map_k, k, c.n_tokens, c.n_kv_heads, c.n_tokens, 128))
-    return MEDA_ERR_CUDA;
-  StatsPolicy::Params prm;
+  CUtensorMap map_k;
+  if (!make_rows_map(ctx, &map_k, k, c.n_tokens, c.n_kv_heads, c.n_tokens, 128)) return MEDA_ERR_CUDA;
+  WinStatsParams prm;
+  prm.q = static_cast<const __nv_bfloat16*>(q_win);
   prm.modality = ctx->ws.modality;
+  prm.tile_class = ctx->ws.tile_class;
   prm.partial = ctx->ws.stats_partial;
+  prm.row_stats = row_stats;
+  prm.coef_vis = ctx->ws.coef_vis;
+  prm.coef_text = ctx->ws.coef_text;
+  prm.counters = ctx->ws.stats_counters;
   prm.n = c.n_tokens; prm.hq = c.n_q_heads; prm.group = ctx->group; prm.w = c.window;
   prm.cols = ctx->group * c.window;
   prm.row_blocks = (prm.cols + 255) / 256;
@@ -226,14 +235,7 @@ meda_status launch_stats_fast(meda_ctx* ctx, const void* q_win, const void* k, f
   const int items = c.n_kv_heads * prm.row_blocks * prm.chunks;
   {
     LaunchScope scope(ctx, MEDA_K_STATS, st);
-    umma_stream_kernel<StatsPolicy><<<std::min(items, ctx->sm_count), us_threads<StatsPolicy>(), StreamShared<StatsPolicy>::alloc, st>>>(
-        map_q, map_k, prm, ctx->ws.status);
-  }
-  {
-    LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
-    stats_combine_kernel<<<(c.n_q_heads * c.window + 7) / 8, 256, 0, st>>>(ctx->ws.stats_partial, row_stats,
-                                                                               prm.chunks * StatsPolicy::kEpilogueGroups,
-                                                                               c.n_q_heads * c.window);
+    window_stats_kernel<<<std::min(items, ctx->sm_count), kWsThreads, WinStatsSmem::alloc, st>>>(map_k, prm, ctx->ws.status);
   }
   return launch_status();
 }
@@ -263,8 +265,10 @@ meda_status raise_sweep_smem() {
                               (int)StreamShared<SweepPolicy<W, MODE>>::alloc) == cudaSuccess ? MEDA_OK : MEDA_ERR_CUDA;
 }
 
+// `coef_ready`: the per-column constants were written by the normaliser sweep that ran just before on this
+// stream; otherwise (row_stats handed in by the caller) they are derived from row_stats first.
 meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
-                              float* scores, float* entropy, cudaStream_t st) {
+                              float* scores, float* entropy, bool coef_ready, cudaStream_t st) {
   const meda_config& c = ctx->cfg;
   if (((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(q_win)) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
   CUtensorMap map_q, map_k;
@@ -272,7 +276,7 @@ meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, c
       !make_rows_map(ctx, &map_k, k, c.n_tokens, c.n_kv_heads, c.n_tokens, 128))
     return MEDA_ERR_CUDA;
   const int rows = c.n_q_heads * c.window;
-  {
+  if (!coef_ready) {
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
     sweep_coef_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_stats, ctx->ws.coef_vis, ctx->ws.coef_text, rows,
                                                           (float)c.n_q_heads);
@@ -807,14 +811,32 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   // the partial normalisers also serve the visual query window of meda_layer_entropy (up to kMaxWindow rows)
   if (st == MEDA_OK)
     st = carve(&ws.stats_partial,
-               std::max((int64_t)std::max(kStatsChunks, ctx->stats_chunks * StatsPolicy::kEpilogueGroups) * c.n_q_heads * c.window * 4,
+               std::max((int64_t)std::max(kStatsChunks, ctx->stats_chunks) * c.n_q_heads * c.window * 4,
                         (int64_t)kStatsChunks * c.n_q_heads * kMaxWindow * 4), &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.row_stats_vis, (int64_t)c.n_q_heads * kMaxWindow * 4, &ws.bytes);
   if (ctx->fast_attn) {
     if (st == MEDA_OK) st = carve(&ws.coef_vis, (int64_t)c.n_q_heads * c.window, &ws.bytes);
     if (st == MEDA_OK) st = carve(&ws.coef_text, (int64_t)c.n_q_heads * c.window, &ws.bytes);
-    if (st == MEDA_OK && cudaFuncSetAttribute(umma_stream_kernel<StatsPolicy>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)StreamShared<StatsPolicy>::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
+    if (st == MEDA_OK && cudaFuncSetAttribute(window_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)WinStatsSmem::alloc) != cudaSuccess) st = MEDA_ERR_CUDA;
+    // one class byte per 32-key chunk (0 all text, 1 all visual, 2 mixed or past the end), four per 128-key tile
+    const int64_t n_tiles128 = (n + 127) / 128;
+    std::vector<uint32_t> tile_class((size_t)n_tiles128, 0u);
+    for (int64_t ch = 0; ch < n_tiles128 * 4; ++ch) {
+      uint32_t cls = 2u;
+      if (ch * 32 + 32 <= n) {
+        int vis = 0;
+        for (int x = 0; x < 32; ++x) vis += modality[(size_t)(ch * 32 + x)] == MEDA_VISUAL;
+        cls = vis == 32 ? 1u : (vis == 0 ? 0u : 2u);
+      }
+      tile_class[(size_t)(ch / 4)] |= cls << (8 * (ch % 4));
+    }
+    if (st == MEDA_OK) st = carve(&ws.tile_class, n_tiles128, &ws.bytes);
+    if (st == MEDA_OK && cudaMemcpy(ws.tile_class, tile_class.data(), (size_t)n_tiles128 * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+      st = MEDA_ERR_CUDA;
+    ctx->stats_counter_count = (int)(hkv * ((ctx->group * c.window + 255) / 256) * kWsEpilogueWarps);
+    if (st == MEDA_OK) st = carve(&ws.stats_counters, ctx->stats_counter_count, &ws.bytes);
+    if (st == MEDA_OK && cudaMemset(ws.stats_counters, 0, (size_t)ctx->stats_counter_count * 4) != cudaSuccess) st = MEDA_ERR_CUDA;
     if (st == MEDA_OK) st = raise_sweep_smem<32, 0>();
     if (st == MEDA_OK) st = raise_sweep_smem<32, 1>();
     if (st == MEDA_OK) st = raise_sweep_smem<64, 0>();
@@ -953,7 +975,12 @@ meda_status meda_poll_status(meda_ctx* ctx, void* stream) {
   int code = 0;
   MEDA_CUDA_TRY(cudaStreamSynchronize(as_stream(stream)));
   MEDA_CUDA_TRY(cudaMemcpy(&code, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost));
-  if (code != 0) MEDA_CUDA_TRY(cudaMemset(ctx->ws.status, 0, sizeof(int)));
+  if (code != 0) {
+    MEDA_CUDA_TRY(cudaMemset(ctx->ws.status, 0, sizeof(int)));
+    // a kernel that gave up may have left its completion counters mid-count
+    if (ctx->ws.stats_counters)
+      MEDA_CUDA_TRY(cudaMemset(ctx->ws.stats_counters, 0, (size_t)ctx->stats_counter_count * sizeof(unsigned int)));
+  }
   return (meda_status)code;
 }
 
@@ -970,7 +997,7 @@ meda_status meda_window_scores(meda_ctx* ctx, int32_t layer, const void* q_win, 
   meda_status r;
   if (ctx->fast_attn) {
     r = launch_stats_fast(ctx, q_win, k, row_stats, st);
-    if (r == MEDA_OK) r = launch_sweep_fast(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+    if (r == MEDA_OK) r = launch_sweep_fast(ctx, layer, q_win, k, row_stats, scores, entropy, true, st);
   } else if (ctx->cfg.dtype == MEDA_F32) {
     r = launch_stats<float>(ctx, q_win, k, row_stats, st);
     if (r == MEDA_OK) r = launch_sweep<float>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
@@ -985,7 +1012,7 @@ meda_status meda_window_scores_from_stats(meda_ctx* ctx, int32_t layer, const vo
                                           const float* row_stats, float* scores, float* entropy, void* stream) {
   if (!layer_ok(ctx, layer) || !q_win || !k || !row_stats || !scores) return MEDA_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
-  if (ctx->fast_attn) return launch_sweep_fast(ctx, layer, q_win, k, row_stats, scores, entropy, st);
+  if (ctx->fast_attn) return launch_sweep_fast(ctx, layer, q_win, k, row_stats, scores, entropy, false, st);
   if (ctx->cfg.dtype == MEDA_F32) return launch_sweep<float>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
   return launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, scores, entropy, st);
 }
@@ -1015,7 +1042,7 @@ meda_status meda_layer_entropy(meda_ctx* ctx, int32_t layer, const void* q_win, 
   cudaStream_t st = as_stream(stream);
   meda_status r = MEDA_OK;
   if (q_win) {
-    if (ctx->fast_attn) r = launch_sweep_fast(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
+    if (ctx->fast_attn) r = launch_sweep_fast(ctx, layer, q_win, k, row_stats, nullptr, entropy, false, st);
     else if (ctx->cfg.dtype == MEDA_F32) r = launch_sweep<float>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
     else r = launch_sweep<__nv_bfloat16>(ctx, layer, q_win, k, row_stats, nullptr, entropy, st);
   }

@@ -20,6 +20,8 @@ struct Workspace {
   uint8_t* modality = nullptr;        // [n padded to a multiple of 256, + 128] 0 = text, 1 = visual, 2 = padding
   float2* coef_vis = nullptr;         // [Hq * w] per-column constants of the tensor-core scores sweep
   float2* coef_text = nullptr;        // [Hq * w]
+  uint32_t* tile_class = nullptr;     // [ceil(n / 128)] one class byte per 32-key chunk: 0 text, 1 visual, 2 mixed / padding
+  unsigned int* stats_counters = nullptr;   // completion counters of the normaliser sweep's row sets, zero between launches
   int* status = nullptr;              // device status word (first error wins)
   float* stats_partial = nullptr;     // [chunks][Hq][w][4]
   float* row_stats_vis = nullptr;     // [Hq][<= kMaxWindow][4] normalisers of the visual query window (E_VT)
@@ -73,6 +75,7 @@ struct meda_ctx {
   int select_cluster = 0;        // blocks per thread-block cluster (one cluster per KV head) of the selection; 0: single-block kernel
   int stats_chunks = 0;   // key chunks of the tensor-core normaliser sweep
   int stats_tiles_per_chunk = 0;
+  int stats_counter_count = 0;
   void* encode_tiled = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
   meda::Workspace ws;
 };

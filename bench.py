@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--no-prompt-scores", action="store_true",
                     help="skip the context measurement of Eq. 8 taken over every prompt row (one layer)")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--oracle-whole-pass", action="store_true",
+                    help="time the oracle on the whole pass, un-sampled, whatever its size (minutes for the large workloads)")
     return ap.parse_args()
 
 
@@ -59,42 +61,89 @@ def peaks():
 # CPU oracle leg (cpu_baseline and --impl reference)
 # ------------------------------------------------------------------------------------------------
 
-def oracle_sample_seconds(wl, layer=0):
-    """Times the oracle, as it stands, on a bounded sample of the workload: one layer, KV head 0
-    with its query heads: scores + entropy of that head group, selection of that head at the uniform
-    budget rho * n, and merging of every `stride`-th less-important row (stride > 1 only for long
-    prompts; the merge time is multiplied back by the stride).  Returns (seconds, description)."""
+WHOLE_PASS_MAX_SIMILARITIES = 2.5e9     # below this many similarity entries the oracle runs the whole pass, un-sampled
+
+
+def uniform_budgets(wl):
+    """Budget rows (S, M, N) when no device run is at hand: every layer gets rho * n."""
+    s = max(wl.min_budget, int(round(wl.rho * wl.n_tokens)))
+    return [(s, (s * 3) // 4, s - (s * 3) // 4)] * wl.n_layers
+
+
+def similarity_entries(wl, budgets):
+    """(n - S_l) * S_l summed over layers and KV heads: the size of the oracle's dominant step."""
+    return float(sum((wl.n_tokens - s) * s for s, _, _ in budgets)) * wl.n_kv_heads
+
+
+def oracle_whole_pass_seconds(wl):
+    """The oracle's whole pass (compress_pass: every layer, every head, nothing sampled), timed as it stands."""
+    import torch
+    from oracle import meda_oracle as O
+    from paper_2502_17599_b200 import workloads as W
+    layers = [tuple(t.to(torch.float64).numpy() for t in W.make_layer(wl, l, "cpu")) for l in range(wl.n_layers)]
+    mod = wl.modality().numpy()
+    t0 = time.perf_counter()
+    O.compress_pass(layers, mod, wl.global_budget, wl.min_budget, wl.dtype)
+    return time.perf_counter() - t0, "whole pass, every layer and head, un-sampled"
+
+
+def oracle_sample_seconds(wl, budgets=None, whole_pass=False):
+    """Times the oracle, as it stands, on a bounded sample of the workload and scales it to the whole pass.
+
+    `budgets`: the (S, M, N) rows of the measured run (read back from the device), so that the sample has a
+    budget the pass really has; without them (reference arm, no device) a uniform rho * n is assumed and said so.
+    The sample is one layer (the one whose (n - S) S is closest to the mean over layers, i.e. a typical share of
+    the dominant similarity step), KV head 0 with its query heads: scores + entropy of that head group, selection
+    of that head at the layer's (M, N), and merging of every `stride`-th less-important row.  Scaling: phase A and
+    selection x (KV heads x layers); the merge by the ratio of similarity entries, whole pass / sampled.
+    Returns (seconds for the whole pass, description, extrapolated flag)."""
     import numpy as np
     import torch
     from oracle import meda_oracle as O
     from paper_2502_17599_b200 import workloads as W
 
+    real = budgets is not None
+    rows = [tuple(int(x) for x in b) for b in budgets] if real else uniform_budgets(wl)
+    n = wl.n_tokens
+    if whole_pass or (similarity_entries(wl, rows) <= WHOLE_PASS_MAX_SIMILARITIES and wl.n_layers * n <= 1.2e6):
+        sec, desc = oracle_whole_pass_seconds(wl)
+        return sec, desc, False
+    work = [(n - s) * s for s, _, _ in rows]
+    mean_work = sum(work) / len(work)
+    layer = min(range(len(rows)), key=lambda l: abs(work[l] - mean_work))
+    s, m, n_imp = rows[layer]
     g = wl.n_q_heads // wl.n_kv_heads
-    sub = wl.with_(n_layers=max(layer + 1, 1))
+    sub = wl.with_(n_layers=layer + 1)
     q, k, v = W.make_layer(sub, layer, "cpu")
     qh = q[:g].to(torch.float64).numpy()
     kh = k[:1].to(torch.float64).numpy()
     vh = v[:1].to(torch.float64).numpy()
     mod = wl.modality().numpy()
-    s = max(wl.min_budget, int(round(wl.rho * wl.n_tokens)))
-    m = (s * 3) // 4
-    stride = max(1, wl.n_tokens // 16384)
+    # bound the merge sample to about 4e8 similarity entries (a few seconds of fp64 matmul and normalisation)
+    stride = max(1, int(np.ceil((n - s) * s / 4e8)))
     t0 = time.perf_counter()
     a_s = O.window_scores(qh, kh)
     O.cross_modal_entropy(qh, kh, mod)
-    conserved, less = O.select_topk(a_s[0], mod, m, s - m)
+    conserved, less = O.select_topk(a_s[0], mod, m, n_imp)
     t1 = time.perf_counter()
-    km, vm, counts, target = O.merge_kv(kh[0], vh[0], conserved, less[::stride])
+    sampled = less[::stride]
+    km, vm, counts, target = O.merge_kv(kh[0], vh[0], conserved, sampled)
     O.round_to_dtype(km, wl.dtype), O.round_to_dtype(vm, wl.dtype)
     t2 = time.perf_counter()
-    dt = (t1 - t0) + stride * (t2 - t1)
-    return dt, (f"layer {layer}, KV head 0 of {wl.n_kv_heads} ({g} query heads), uniform budget S={s}, merge on every "
-                f"{stride}-th less-important row with its time x{stride}; extrapolated x{wl.n_kv_heads} heads")
+    per_head_layer = t1 - t0
+    merge_scale = similarity_entries(wl, rows) / max(float(sampled.size) * s, 1.0)
+    total = per_head_layer * wl.n_kv_heads * wl.n_layers + (t2 - t1) * merge_scale
+    desc = (f"layer {layer}, KV head 0 of {wl.n_kv_heads} ({g} query heads), "
+            f"{'budget row of the measured run' if real else 'uniform budget rho*n (no device run at hand)'} "
+            f"(S, M, N) = ({s}, {m}, {n_imp}); phase A + selection timed once and x{wl.n_kv_heads * wl.n_layers} "
+            f"(heads x layers); merge timed on every {stride}-th less-important row ({sampled.size} x {s} similarities) "
+            f"and scaled x{merge_scale:.1f} to the pass's {similarity_entries(wl, rows):.3g} similarities")
+    return total, desc, True
 
 
 def oracle_throughput(wl, seconds):
-    # one KV head of one layer took `seconds`: a whole layer-pass takes n_kv_heads times that
-    return wl.n_tokens / (seconds * wl.n_kv_heads)
+    # `seconds` is the (measured or extrapolated) time of the whole pass
+    return wl.n_layers * wl.n_tokens / seconds
 
 
 def cpu_threads():
@@ -116,9 +165,9 @@ def run_reference(args):
         wl = wl.with_(name=f"{wl.name}_first{args.layers}layers", n_layers=min(args.layers, wl.n_layers))
     import numpy  # noqa: F401  (loads BLAS before the thread count is read)
     times = []
-    desc = ""
+    desc, extrapolated = "", False
     for i in range(args.warmup + args.steps):
-        dt, desc = oracle_sample_seconds(wl)
+        dt, desc, extrapolated = oracle_sample_seconds(wl, whole_pass=args.oracle_whole_pass)
         if i >= args.warmup:
             times.append(dt)
     sec = sum(times) / len(times)
@@ -128,7 +177,8 @@ def run_reference(args):
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "shape": wl.description, "sample": desc},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
+                         "extrapolated": extrapolated},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -482,9 +532,9 @@ def run_ours(args):
 
     cpu = None
     if not args.no_cpu_baseline:
-        sec, desc = oracle_sample_seconds(wl)
+        sec, desc, extrapolated = oracle_sample_seconds(wl, cp.budgets.cpu().numpy(), whole_pass=args.oracle_whole_pass)
         cpu = {"value": oracle_throughput(wl, sec), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-               "sample": desc, "sample_seconds": sec}
+               "sample": desc, "pass_seconds": sec, "extrapolated": extrapolated}
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -21,6 +21,7 @@
 #include "prompt_scores_sm100.cuh"
 #include "select.cuh"
 #include "window_stats_sm100.cuh"
+#include "window_sweep_sm100.cuh"
 
 using namespace meda;
 
@@ -62,6 +63,7 @@ void free_workspace(Workspace& ws) {
   cudaFree(ws.coef_text);
   cudaFree(ws.tile_class);
   cudaFree(ws.stats_counters);
+  cudaFree(ws.sweep_counter);
   for (int i = 0; i < 2; ++i) { cudaFree(ws.sort_keys[i]); cudaFree(ws.sort_rows[i]); }
   cudaFree(ws.sort_table);
   cudaFree(ws.seg_start);
@@ -265,14 +267,48 @@ meda_status raise_sweep_smem() {
                               (int)StreamShared<SweepPolicy<W, MODE>>::alloc) == cudaSuccess ? MEDA_OK : MEDA_ERR_CUDA;
 }
 
+// The scores + entropy sweep for KV groups of 129 .. 256 query rows (grouped-query attention): one launch that
+// also finishes the entropy.
+template <int W, int MODE>
+void launch_window_sweep(meda_ctx* ctx, const CUtensorMap& map_k, const CUtensorMap& map_q, const float* row_stats,
+                         float* scores, float* entropy_out, cudaStream_t st) {
+  const meda_config& c = ctx->cfg;
+  WinSweepParams prm;
+  prm.modality = ctx->ws.modality;
+  prm.vis = ctx->ws.coef_vis;
+  prm.text = ctx->ws.coef_text;
+  prm.row_stats = row_stats;
+  prm.scores = scores;
+  prm.ent_partial = entropy_out ? ctx->ws.ent_partial : nullptr;
+  prm.entropy_out = entropy_out;
+  prm.done_counter = ctx->ws.sweep_counter;
+  prm.n = c.n_tokens; prm.hkv = c.n_kv_heads; prm.cols = ctx->group * c.window;
+  prm.n_blocks = (c.n_tokens + 255) / 256;
+  prm.a_stages = win_sweep_a_stages(prm.cols);
+  prm.sc2 = kLog2e / sqrtf((float)c.head_dim);
+  prm.ln_hq = logf((float)c.n_q_heads);
+  const WinSweepSmem L(prm.cols, prm.a_stages);
+  window_sweep_kernel<W, MODE><<<std::min(prm.n_blocks, ctx->sm_count), kSwThreads, L.alloc(), st>>>(map_k, map_q, prm,
+                                                                                                    ctx->ws.status);
+}
+
+template <int W, int MODE>
+meda_status raise_window_sweep_smem() {
+  return cudaFuncSetAttribute(window_sweep_kernel<W, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) ==
+                 cudaSuccess ? MEDA_OK : MEDA_ERR_CUDA;
+}
+
 // `coef_ready`: the per-column constants were written by the normaliser sweep that ran just before on this
 // stream; otherwise (row_stats handed in by the caller) they are derived from row_stats first.
 meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, const void* k, const float* row_stats,
                               float* scores, float* entropy, bool coef_ready, cudaStream_t st) {
   const meda_config& c = ctx->cfg;
   if (((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(q_win)) & 15u) != 0) return MEDA_ERR_INVALID_ARG;
+  const int cols = ctx->group * c.window;
+  const bool grouped = ctx->fast_sweep_grouped;     // the kernel for several query heads per KV head
   CUtensorMap map_q, map_k;
-  if (!make_rows_map(ctx, &map_q, q_win, (int64_t)c.n_q_heads * c.window, 1, (int64_t)c.n_q_heads * c.window, 128) ||
+  if (!make_rows_map(ctx, &map_q, q_win, (int64_t)c.n_q_heads * c.window, 1, (int64_t)c.n_q_heads * c.window,
+                     grouped ? (uint32_t)cols : 128u) ||
       !make_rows_map(ctx, &map_k, k, c.n_tokens, c.n_kv_heads, c.n_tokens, 128))
     return MEDA_ERR_CUDA;
   const int rows = c.n_q_heads * c.window;
@@ -280,6 +316,13 @@ meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, c
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
     sweep_coef_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_stats, ctx->ws.coef_vis, ctx->ws.coef_text, rows,
                                                           (float)c.n_q_heads);
+  }
+  if (grouped) {
+    LaunchScope scope(ctx, MEDA_K_SWEEP, st);
+    float* e_out = entropy ? entropy + layer : nullptr;
+    if (c.entropy_mode == 0) launch_window_sweep<32, 0>(ctx, map_k, map_q, row_stats, scores, e_out, st);
+    else launch_window_sweep<32, 1>(ctx, map_k, map_q, row_stats, scores, e_out, st);
+    return launch_status();
   }
   {
     LaunchScope scope(ctx, MEDA_K_SWEEP, st);
@@ -779,7 +822,10 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   }
   ctx->fast = c.dtype == MEDA_BF16 && c.head_dim == kFastDim;
   ctx->fast_attn = ctx->fast && (c.window == 32 || c.window == 64) && ctx->group * c.window <= kSweepMaxCols;
-  ctx->ent_slots = std::max(generic_tiles(c.n_tokens), ((c.n_tokens + 255) / 256) * kUsEpilogueWarps);
+  const int cols_per_group = ctx->group * c.window;
+  // (window 32 only: with 64 rows the kernel's per-thread state does not fit its registers)
+  ctx->fast_sweep_grouped = ctx->fast_attn && c.window == 32 && cols_per_group > 128 && cols_per_group <= kSwMaxCols;
+  ctx->ent_slots = std::max(generic_tiles(c.n_tokens), ((c.n_tokens + 255) / 256) * kSwEpilogueWarps);
   {
     // Key chunks of the tensor-core normaliser sweep.  An item = (KV head, row block, key chunk); the grid is
     // one block per SM, so a launch takes ceil(items / SMs) waves of (tiles per chunk + about 1.5 tiles of
@@ -841,6 +887,10 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     if (st == MEDA_OK) st = raise_sweep_smem<32, 1>();
     if (st == MEDA_OK) st = raise_sweep_smem<64, 0>();
     if (st == MEDA_OK) st = raise_sweep_smem<64, 1>();
+    if (st == MEDA_OK) st = raise_window_sweep_smem<32, 0>();
+    if (st == MEDA_OK) st = raise_window_sweep_smem<32, 1>();
+    if (st == MEDA_OK) st = carve(&ws.sweep_counter, 1, &ws.bytes);
+    if (st == MEDA_OK && cudaMemset(ws.sweep_counter, 0, 4) != cudaSuccess) st = MEDA_ERR_CUDA;
   }
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.decode_partial, (int64_t)c.n_q_heads * kDecSplits * (c.head_dim + 2), &ws.bytes);
@@ -980,6 +1030,7 @@ meda_status meda_poll_status(meda_ctx* ctx, void* stream) {
     // a kernel that gave up may have left its completion counters mid-count
     if (ctx->ws.stats_counters)
       MEDA_CUDA_TRY(cudaMemset(ctx->ws.stats_counters, 0, (size_t)ctx->stats_counter_count * sizeof(unsigned int)));
+    if (ctx->ws.sweep_counter) MEDA_CUDA_TRY(cudaMemset(ctx->ws.sweep_counter, 0, sizeof(unsigned int)));
   }
   return (meda_status)code;
 }

@@ -21,6 +21,7 @@ struct Workspace {
   float2* coef_vis = nullptr;         // [Hq * w] per-column constants of the tensor-core scores sweep
   float2* coef_text = nullptr;        // [Hq * w]
   uint32_t* tile_class = nullptr;     // [ceil(n / 128)] one class byte per 32-key chunk: 0 text, 1 visual, 2 mixed / padding
+  unsigned int* sweep_counter = nullptr;    // blocks of the grouped scores sweep that have finished, zero between launches
   unsigned int* stats_counters = nullptr;   // completion counters of the normaliser sweep's row sets, zero between launches
   int* status = nullptr;              // device status word (first error wins)
   float* stats_partial = nullptr;     // [chunks][Hq][w][4]
@@ -72,6 +73,7 @@ struct meda_ctx {
   int sort_passes = 1;    // 9-bit digit passes needed to order slots < n_tokens
   bool fast = false;      // bf16 with head_dim 128: tensor-core kernels are used
   bool fast_attn = false; // ... and window 32 or 64: phase A runs on the tensor cores too
+  bool fast_sweep_grouped = false;   // ... and 129 .. 256 query rows per KV head: the grouped scores sweep
   int select_cluster = 0;        // blocks per thread-block cluster (one cluster per KV head) of the selection; 0: single-block kernel
   int stats_chunks = 0;   // key chunks of the tensor-core normaliser sweep
   int stats_tiles_per_chunk = 0;

@@ -100,8 +100,9 @@ def test_tensor_core_kernels_keep_tensor_memory_loads_out_of_local_memory():
     assert res.returncode == 0, res.stderr
     lines = (res.stdout + res.stderr).splitlines()
     hits = [i for i, line in enumerate(lines)
-            if "Function properties" in line and ("nearest_kernel" in line or "umma_stream_kernel" in line)]
-    assert len(hits) >= 6, "tensor-core kernels not found in the ptxas report"
+            if "Function properties" in line and any(name in line for name in (
+                "nearest_kernel", "umma_stream_kernel", "window_stats_kernel", "window_sweep_kernel"))]
+    assert len(hits) >= 9, "tensor-core kernels not found in the ptxas report"
     for i in hits:
         assert "0 bytes spill stores, 0 bytes spill loads" in lines[i + 1], (lines[i], lines[i + 1])
 

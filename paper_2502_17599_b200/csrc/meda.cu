@@ -836,7 +836,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     const int per_chunk_items = std::max(1, c.n_kv_heads * row_blocks);
     int want = 1;
     double best = 1e300;
-    for (int cand = 1; cand <= tiles && cand * per_chunk_items <= 4 * ctx->sm_count; ++cand) {
+    for (int cand = 1; cand <= tiles && cand <= kWsMaxChunks && cand * per_chunk_items <= 4 * ctx->sm_count; ++cand) {
       const int tpc = (tiles + cand - 1) / cand;
       const int chunks = (tiles + tpc - 1) / tpc;
       const int waves = (chunks * per_chunk_items + ctx->sm_count - 1) / ctx->sm_count;
@@ -857,7 +857,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   // the partial normalisers also serve the visual query window of meda_layer_entropy (up to kMaxWindow rows)
   if (st == MEDA_OK)
     st = carve(&ws.stats_partial,
-               std::max((int64_t)std::max(kStatsChunks, ctx->stats_chunks) * c.n_q_heads * c.window * 4,
+               std::max((int64_t)std::max(kStatsChunks, (ctx->stats_chunks + 7) / 8 * 8) * c.n_q_heads * c.window * 4,
                         (int64_t)kStatsChunks * c.n_q_heads * kMaxWindow * 4), &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.row_stats_vis, (int64_t)c.n_q_heads * kMaxWindow * 4, &ws.bytes);
   if (ctx->fast_attn) {

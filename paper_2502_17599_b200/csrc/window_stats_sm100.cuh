@@ -40,13 +40,14 @@ constexpr uint32_t kWsStageBytes = 2 * kUsHalfTile;       // 128 keys x 128 dims
 constexpr uint32_t kWsTmemCols = 512;
 constexpr uint32_t kWsAccBase = 128;                      // columns [0, 128): the query rows, 64 per row tile
 constexpr uint32_t kWsSlots = 3;                          // accumulator slots of 128 columns
+constexpr int kWsMaxChunks = 64;                          // key runs per (KV group, row block): at most this many partials per row
 constexpr int kWsPolyOf8 = 2;                             // exponentials per 8 that take the FMA pipes
 
 struct WinStatsParams {
   const __nv_bfloat16* q;        // [Hq * w][128]: window rows, head-major
   const uint8_t* modality;       // padded to a multiple of 128 with the value 2 (= no key)
   const uint32_t* tile_class;    // per 128-key tile: one byte per 32-key chunk: 0 all text, 1 all visual, 2 mixed / padding
-  float* partial;                // [chunks][Hq][w][4]
+  float* partial;                // [Hq * w][chunks_pad][4]: a row's partials are contiguous (chunks_pad = chunks rounded up to 8)
   float* row_stats;              // [Hq][w][4]  (written by the merging warps)
   float2* coef_vis;              // [Hq * w]    per-column constants of the second sweep, or null
   float2* coef_text;             // [Hq * w]
@@ -169,12 +170,19 @@ struct WinStatsRow {
 // load may be in flight in the calling thread (a register that is saved around the call must hold its value).
 __device__ __noinline__ WinStatsRow win_stats_mixed_chunk(WinStatsRow s, const float* logits, float sc2, const uint8_t* mod32,
                                                           int j0, int last_visible) {
-#pragma unroll 1
-  for (int x = 0; x < 32; ++x) {
-    const int md = mod32[x];
-    if (md < 2 && j0 + x <= last_visible) {
-      if (md == MEDA_VISUAL) WinStatsRow::absorb(s.mv, s.zv, logits[x] * sc2);
-      else WinStatsRow::absorb(s.mt, s.zt, logits[x] * sc2);
+  // the chunk's 32 modality bytes in two loads (the map is padded and a chunk starts on a multiple of 32)
+  const uint4 ma = __ldg(reinterpret_cast<const uint4*>(mod32)), mb = __ldg(reinterpret_cast<const uint4*>(mod32) + 1);
+  const uint32_t mw[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+#pragma unroll
+  for (int w8 = 0; w8 < 8; ++w8) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int x = 4 * w8 + b;
+      const int md = (int)((mw[w8] >> (8 * b)) & 0xffu);
+      if (md < 2 && j0 + x <= last_visible) {
+        if (md == MEDA_VISUAL) WinStatsRow::absorb(s.mv, s.zv, logits[x] * sc2);
+        else WinStatsRow::absorb(s.mt, s.zt, logits[x] * sc2);
+      }
     }
   }
   return s;
@@ -186,19 +194,37 @@ __device__ __noinline__ WinStatsRow win_stats_mixed_chunk(WinStatsRow s, const f
 //   text = (m_all * log2e,                     1 / z_all)                                 for text keys
 // (a row that sees no visual key gets (+huge, 0): its exponentials are 0).
 __device__ __forceinline__ void win_stats_finish_row(const WinStatsParams& p, int h, int i) {
-  const size_t row = (size_t)h * p.w + i, rows = (size_t)p.hq * p.w;
-  const float4* part = reinterpret_cast<const float4*>(p.partial) + row;
+  const size_t row = (size_t)h * p.w + i;
+  const int chunks_pad = (p.chunks + 7) / 8 * 8;
+  const float4* part = reinterpret_cast<const float4*>(p.partial) + row * chunks_pad;
+  // The row's partials lie in a few consecutive 128-byte lines, written by other blocks (this block has not read
+  // them before, and the first-level cache holds nothing from earlier launches).  One load per line goes out first,
+  // so that all lines travel at once; the rest of each line then comes at cache speed.  Each line's eight partials
+  // are merged as a fixed tree and the lines in order: the dependent chain is a few merges long instead of one per
+  // key run, and the result depends on nothing but the data.
+  constexpr int kLines = (kWsMaxChunks + 7) / 8;
+  const float4 nothing = make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
+  float4 head[kLines];
+#pragma unroll
+  for (int b = 0; b < kLines; ++b) head[b] = (8 * b < p.chunks) ? part[8 * b] : nothing;
   float m = -INFINITY, z = 0.f, mv = -INFINITY, zv = 0.f;
-  for (int c0 = 0; c0 < p.chunks; c0 += 8) {
-    float4 x[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) x[u] = __ldcg(part + (size_t)min(c0 + u, p.chunks - 1) * rows);   // written by other blocks: L2
+  for (int b = 0; b < kLines; ++b) {
+    if (8 * b < p.chunks) {
+      float4 x[8];
+      x[0] = head[b];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      if (c0 + u < p.chunks) {
-        merge_mz(m, z, x[u].x, x[u].y);
-        merge_mz(mv, zv, x[u].z, x[u].w);
+      for (int u = 1; u < 8; ++u) x[u] = (8 * b + u < p.chunks) ? part[8 * b + u] : nothing;
+#pragma unroll
+      for (int step = 1; step < 8; step <<= 1) {
+#pragma unroll
+        for (int u = 0; u < 8; u += 2 * step) {
+          merge_mz(x[u].x, x[u].y, x[u + step].x, x[u + step].y);
+          merge_mz(x[u].z, x[u].w, x[u + step].z, x[u + step].w);
+        }
       }
+      merge_mz(m, z, x[0].x, x[0].y);
+      merge_mz(mv, zv, x[0].z, x[0].w);
     }
   }
   reinterpret_cast<float4*>(p.row_stats)[row] = make_float4(m, z, mv, zv);
@@ -424,7 +450,7 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
           const float m_all = fmaxf(row.mv, row.mt);
           float z_all = 0.f;
           if (m_all > -INFINITY) z_all = row.zv * fast_exp2(row.mv - m_all) + row.zt * fast_exp2(row.mt - m_all);
-          reinterpret_cast<float4*>(p.partial)[((size_t)it.kc * p.hq + h) * p.w + i_win] =
+          reinterpret_cast<float4*>(p.partial)[((size_t)h * p.w + i_win) * ((p.chunks + 7) / 8 * 8) + it.kc] =
               make_float4(m_all * kLn2, z_all, row.mv * kLn2, row.zv);
         }
         __threadfence();

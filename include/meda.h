@@ -71,8 +71,8 @@ typedef struct {
   int32_t beta_important;
   int32_t min_budget;     /* per-layer floor of S_l (>= 1); n_tokens is the ceiling */
   int32_t entropy_mode;   /* 0: entropy of the head-averaged attention (Sec. 3.2); 1: mean of per-head entropies */
-  int32_t alloc_mode;     /* 0: Eq. 7; 1: uniform shares (Table 5, "w/o dynamic allocation") */
-  int32_t merge_mode;     /* 0: Eq. 12 average merging; 1: drop the less important pairs (Table 5, "w/o merging") */
+  int32_t alloc_mode;     /* 0: Eq. 7; 1: uniform shares (Table 5, the row without dynamic allocation) */
+  int32_t merge_mode;     /* 0: Eq. 12 average merging; 1: drop the less important pairs (Table 5, the row without merging) */
 } meda_config;
 
 /* Creates a context: validates the configuration, uploads the modality map built from

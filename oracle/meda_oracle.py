@@ -135,9 +135,9 @@ def directed_entropy_term(q: np.ndarray, k: np.ndarray, q_pos: np.ndarray, key_s
     """One line of Eq. 5: (1/rows) sum_i sum_j A[i, j] log A[i, j]  (a non-positive number).
 
     A is Eq. 4's cross-modal attention: the softmax is taken over the keys of the *other*
-    modality only (`key_subset`), so every row is a distribution.  entropy_mode 0 (the paper:
-    "A is average attention across multi-heads"): A = mean over the query heads of the
-    per-head softmax, then the row entropies.  entropy_mode 1: the mean over heads of the
+    modality only (`key_subset`), so every row is a distribution.  entropy_mode 0 (Sec. 3.2
+    defines A as the per-head attention averaged over the heads): A = mean over the query heads of
+    the per-head softmax, then the row entropies.  entropy_mode 1: the mean over heads of the
     per-head sums.  Rows with no visible key in the subset are skipped, and 1/rows counts the
     rows used; no usable row gives 0.
     """
@@ -189,9 +189,9 @@ def cross_modal_entropy(q_win: np.ndarray, k: np.ndarray, modality: np.ndarray,
 # --------------------------------------------------------------------------------------
 
 def allocation_weights(entropy: np.ndarray, alloc_mode: int = 0) -> np.ndarray:
-    """softmax over layers of E_CM (Eq. 7 without the L*rho factor).  The text names the rule
-    "inverse entropy softmax" but the formula and the appendix are a direct softmax: higher
-    entropy, larger share.  alloc_mode 1 = the "w/o dynamic allocation" ablation: uniform."""
+    """softmax over layers of E_CM (Eq. 7 without the L*rho factor).  Sec. 3.2's name for the rule
+    suggests an inversion of the entropy, but Eq. 7 and App. A.3 are a direct softmax: higher
+    entropy, larger share; the equations are followed.  alloc_mode 1 = Table 5's ablation row without dynamic allocation: uniform."""
     e = np.asarray(entropy, dtype=np.float64)
     if alloc_mode == 1:
         return np.full(e.shape, 1.0 / e.size)
@@ -342,7 +342,7 @@ def average_merge(x_g: np.ndarray, conserved: np.ndarray, less: np.ndarray, targ
 def merge_kv(k_g: np.ndarray, v_g: np.ndarray, conserved: np.ndarray, less: np.ndarray,
              target: np.ndarray | None = None, merge_mode: int = 0):
     """Merge step for one (layer, KV head).  The similarity uses keys only and the same
-    assignment is applied to the values.  merge_mode 1 = the "w/o average merging" ablation:
+    assignment is applied to the values.  merge_mode 1 = Table 5's ablation row without average merging:
     the less-important pairs are dropped.  Returns (K_c', V_c', counts, target)."""
     if merge_mode == 1:
         return (k_g[conserved].copy(), v_g[conserved].copy(),

@@ -172,8 +172,8 @@ stats_combine_kernel(const float* __restrict__ partial, float* __restrict__ row_
 
 // ---------------------------------------------------------------------------------------------
 // Sweep 2: scores and/or entropy.  grid = key tiles; each block walks all query heads so that the
-// head-averaged visual attention of its keys (Sec. 3.2: "A is average attention across
-// multi-heads") is complete inside the block.  ent_partial[tile] = sum over the tile's visual keys
+// head-averaged visual attention of its keys (Sec. 3.2 defines A as the mean over the heads of the
+// per-head attention) is complete inside the block.  ent_partial[tile] = sum over the tile's visual keys
 // and all window rows of a log a (entropy_mode 0) or of the head mean of p log p (mode 1).
 // ---------------------------------------------------------------------------------------------
 template <typename T>

@@ -825,7 +825,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   const int cols_per_group = ctx->group * c.window;
   // (window 32 only: with 64 rows the kernel's per-thread state does not fit its registers)
   ctx->fast_sweep_grouped = ctx->fast_attn && c.window == 32 && cols_per_group > 128 && cols_per_group <= kSwMaxCols;
-  ctx->ent_slots = std::max(generic_tiles(c.n_tokens), ((c.n_tokens + 255) / 256) * kSwEpilogueWarps);
+  ctx->ent_slots = std::max(generic_tiles(c.n_tokens), ((c.n_tokens + 127) / 128) * kSwEpilogueWarps);
   {
     // Key chunks of the tensor-core normaliser sweep.  An item = (KV head, row block, key chunk); the grid is
     // one block per SM, so a launch takes ceil(items / SMs) waves of (tiles per chunk + about 1.5 tiles of
@@ -836,7 +836,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     const int per_chunk_items = std::max(1, c.n_kv_heads * row_blocks);
     int want = 1;
     double best = 1e300;
-    for (int cand = 1; cand <= tiles && cand <= kWsMaxChunks && cand * per_chunk_items <= 4 * ctx->sm_count; ++cand) {
+    for (int cand = 1; cand <= tiles && cand * per_chunk_items <= 4 * ctx->sm_count; ++cand) {
       const int tpc = (tiles + cand - 1) / cand;
       const int chunks = (tiles + tpc - 1) / tpc;
       const int waves = (chunks * per_chunk_items + ctx->sm_count - 1) / ctx->sm_count;

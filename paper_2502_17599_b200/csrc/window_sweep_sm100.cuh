@@ -43,7 +43,7 @@ struct WinSweepParams {
   const float2* text;          // [Hq * w]
   const float* row_stats;      // [Hq][w][4] (the entropy's row count comes from it)
   float* scores;               // [Hkv][n] or null
-  float* ent_partial;          // [n_blocks * 16] or null
+  float* ent_partial;          // [ceil(n / 128) * 16] or null: one slot per 128-key tile and epilogue warp
   float* entropy_out;          // entropy[layer] or null
   unsigned int* done_counter;  // zero between launches
   int n, hkv, cols;            // cols = group * W
@@ -72,6 +72,31 @@ struct WinSweepSmem {
 };
 
 __host__ __device__ inline int win_sweep_a_stages(int cols) { return cols <= 224 ? 3 : 2; }
+
+// Work of one block of the grid, in order.  Whole 256-key blocks are dealt round-robin while every block of the
+// grid gets one; the blocks left over for a last, partial round are dealt out in halves (one 128-key tile each),
+// so that the grid ends within half a block of each other instead of a whole one.
+struct WinSweepItem {
+  int blk;        // 256-key block
+  int t0, nt;     // first key tile of the block this item covers, and how many (0: nothing, skip)
+};
+__device__ __forceinline__ bool win_sweep_item(const WinSweepParams& p, int it, WinSweepItem& o) {
+  const int grid = (int)gridDim.x;
+  const int full_rounds = p.n_blocks / grid;
+  if (it < full_rounds) {
+    o.blk = (int)blockIdx.x + it * grid;
+    o.t0 = 0;
+    o.nt = (p.n - o.blk * 256 > 128) ? 2 : 1;
+    return true;
+  }
+  const int left = p.n_blocks - full_rounds * grid;
+  const int h = (int)blockIdx.x + (it - full_rounds) * grid;
+  if (h >= 2 * left) return false;
+  o.blk = full_rounds * grid + h / 2;
+  o.t0 = h & 1;
+  o.nt = (o.t0 == 0 || p.n - o.blk * 256 > 128) ? 1 : 0;
+  return true;
+}
 
 template <int W, int MODE>
 __global__ void __launch_bounds__(kSwThreads, 1)
@@ -129,8 +154,10 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       tma_prefetch_descriptor(&map_q);
       uint32_t a_cnt = 0, b_cnt = 0;
       bool ok = true;
-      for (int blk = blockIdx.x; ok && blk < p.n_blocks; blk += gridDim.x) {
-        const int m_tiles = (p.n - blk * 256 > 128) ? 2 : 1;
+      WinSweepItem item;
+      for (int it = 0; ok && win_sweep_item(p, it, item); ++it) {
+        if (item.nt == 0) continue;
+        const int blk = item.blk;
         for (int g = 0; ok && g < p.hkv; ++g, ++b_cnt) {
           const uint32_t buf = b_cnt & 1u, bphase = (b_cnt >> 1) & 1u;
           ok = mbar_wait(b_empty + buf, bphase ^ 1u, abort_flag);
@@ -141,7 +168,7 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
           bulk_load(c_smem + buf * L.c_bytes, p.vis + (size_t)g * p.cols, (uint32_t)p.cols * 8u, b_full + buf);
           bulk_load(c_smem + buf * L.c_bytes + (uint32_t)p.cols * 8u, p.text + (size_t)g * p.cols, (uint32_t)p.cols * 8u,
                     b_full + buf);
-          for (int t = 0; t < m_tiles; ++t, ++a_cnt) {
+          for (int t = item.t0; t < item.t0 + item.nt; ++t, ++a_cnt) {
             const uint32_t stage = a_cnt % a_stages, aphase = (a_cnt / a_stages) & 1u;
             ok = mbar_wait(a_empty + stage, aphase ^ 1u, abort_flag);
             if (!ok) break;
@@ -160,8 +187,10 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       const uint32_t idesc = umma_idesc_bf16(128, p.cols);
       const uint32_t b_half16 = (L.b_bytes / 2) >> 4;
       bool ok = true;
-      for (int blk = blockIdx.x; ok && blk < p.n_blocks; blk += gridDim.x) {
-        const int m_tiles = (p.n - blk * 256 > 128) ? 2 : 1;
+      WinSweepItem item;
+      for (int it = 0; ok && win_sweep_item(p, it, item); ++it) {
+        if (item.nt == 0) continue;
+        const int m_tiles = item.nt;
         for (int g = 0; ok && g < p.hkv; ++g, ++b_cnt) {
           const uint32_t buf = b_cnt & 1u, bphase = (b_cnt >> 1) & 1u;
           ok = mbar_wait(b_full + buf, bphase, abort_flag);
@@ -217,7 +246,7 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       if (!good) return false;
       tc_fence_after_sync();
       const uint32_t taddr = lane_addr + slot * 256u + (uint32_t)(k * R);
-      float score = 0.f, score2 = 0.f;
+      float score = 0.f;
       auto load = [&](uint32_t (&r)[R], int hl) {
         if constexpr (R == 8) tmem_ld_32x8_issue(taddr + (uint32_t)(hl * W), r);
         else tmem_ld_32x16_issue(taddr + (uint32_t)(hl * W), r);
@@ -238,7 +267,7 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         for (int x = 0; x < R; x += 2) {
           const float4 c = coef[c0 + x / 2];                  // read again rather than kept: registers are short
           score = fmaf(e_prev[x], c.y, score);
-          score2 = fmaf(e_prev[x + 1], c.w, score2);
+          score = fmaf(e_prev[x + 1], c.w, score);
           if (MODE == 0) {
             abar[T][x] = fmaf(e_prev[x], vflag, abar[T][x]);
             abar[T][x + 1] = fmaf(e_prev[x + 1], vflag, abar[T][x + 1]);
@@ -286,7 +315,6 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         }
       }
       if (MODE == 0) consume(((heads - 1) * W + k * R) / 2);
-      score += score2;
       // every column of the unit has been read: hand the accumulators back
       tc_fence_before_sync();
       __syncwarp();
@@ -313,12 +341,16 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     // in front of every unit would stall all sixteen warps for its whole latency.
     const uint8_t* my_mod = p.modality + quarter * 32 + lane;         // the padded map covers whole blocks
     int md_next = 0x0202;                                             // low byte: key tile 0, next byte: key tile 1
-    if ((int)blockIdx.x < p.n_blocks) md_next = my_mod[(size_t)blockIdx.x * 256] | (my_mod[(size_t)blockIdx.x * 256 + 128] << 8);
-    for (int blk = blockIdx.x; ok && blk < p.n_blocks; blk += gridDim.x) {
-      const int m_tiles = (p.n - blk * 256 > 128) ? 2 : 1;
+    WinSweepItem cur;
+    if (win_sweep_item(p, 0, cur)) md_next = my_mod[(size_t)cur.blk * 256] | (my_mod[(size_t)cur.blk * 256 + 128] << 8);
+    for (int it = 0; ok && win_sweep_item(p, it, cur); ++it) {
+      const int blk = cur.blk;
       const int md_pair = md_next;
-      if (blk + (int)gridDim.x < p.n_blocks)
-        md_next = my_mod[(size_t)(blk + gridDim.x) * 256] | (my_mod[(size_t)(blk + gridDim.x) * 256 + 128] << 8);
+      {
+        WinSweepItem nxt;
+        if (win_sweep_item(p, it + 1, nxt)) md_next = my_mod[(size_t)nxt.blk * 256] | (my_mod[(size_t)nxt.blk * 256 + 128] << 8);
+      }
+      if (cur.nt == 0) continue;
       for (int g = 0; ok && g < p.hkv; ++g, ++b_cnt) {
         const uint32_t buf = b_cnt & 1u, bphase = (b_cnt >> 1) & 1u;
         ok = mbar_wait(b_full + buf, bphase, abort_flag);           // the constants have landed
@@ -326,8 +358,8 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         if (!ok) break;
         const float4* cvis = reinterpret_cast<const float4*>(c_smem + buf * L.c_bytes);
         const float4* ctext = reinterpret_cast<const float4*>(c_smem + buf * L.c_bytes + (uint32_t)p.cols * 8u);
-        ok = run_unit(std::integral_constant<int, 0>(), blk, g, md_pair & 0xff, cvis, ctext);
-        if (ok && m_tiles > 1) ok = run_unit(std::integral_constant<int, 1>(), blk, g, md_pair >> 8, cvis, ctext);
+        if (cur.t0 == 0) ok = run_unit(std::integral_constant<int, 0>(), blk, g, md_pair & 0xff, cvis, ctext);
+        if (ok && cur.t0 + cur.nt > 1) ok = run_unit(std::integral_constant<int, 1>(), blk, g, md_pair >> 8, cvis, ctext);
         if (!ok) break;
         __syncwarp();
         if (lane == 0) mbar_arrive(b_empty + buf);                  // this warp no longer reads the constants
@@ -348,7 +380,9 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       plogp = 0.f;
       acc = warp_sum(acc);
       if (p.ent_partial && lane == 0) {
-        p.ent_partial[(size_t)blk * kSwEpilogueWarps + ewarp] = acc;
+        // one slot per 128-key tile and warp: an item's sum goes to its first tile, a zero to its second
+        p.ent_partial[(size_t)(2 * blk + cur.t0) * kSwEpilogueWarps + ewarp] = acc;
+        if (cur.nt > 1) p.ent_partial[(size_t)(2 * blk + 1) * kSwEpilogueWarps + ewarp] = 0.f;
         __threadfence();
       }
     }
@@ -380,7 +414,7 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
   // entropy = -(1 / rows) * sum of the partials, added in a fixed order (thread-strided, then a tree), so that
   // repeated runs give identical bits; rows = window rows that see at least one visual key
   double* red = reinterpret_cast<double*>(smem);         // the key stages are idle by now
-  const int n_partials = p.n_blocks * kSwEpilogueWarps;
+  const int n_partials = ((p.n + 127) / 128) * kSwEpilogueWarps;
   double acc = 0.0;
   for (int e = threadIdx.x; e < n_partials; e += kSwThreads) acc += (double)__ldcg(p.ent_partial + e);
   red[threadIdx.x] = acc;

@@ -166,7 +166,7 @@ def test_full_size_variants_ablation_modes_vision_to_text_term_and_decoding_step
         q, k, v = W.make_layer(wl, l, "cuda")
         qs.append(q); ks.append(k); vs.append(v)
 
-    # ---- "w/o dynamic allocation", "w/o merging", per-head entropies
+    # ---- Table 5's ablation rows: no dynamic allocation, no merging; and per-head entropies
     cp = CompressionPass(wl, entropy_mode=1, alloc_mode=1, merge_mode=1)
     cp.run(qs, ks, vs)
     cp.check()

@@ -836,7 +836,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
     const int per_chunk_items = std::max(1, c.n_kv_heads * row_blocks);
     int want = 1;
     double best = 1e300;
-    for (int cand = 1; cand <= tiles && cand * per_chunk_items <= 4 * ctx->sm_count; ++cand) {
+    for (int cand = 1; cand <= tiles && cand <= kWsMaxChunks && cand * per_chunk_items <= 4 * ctx->sm_count; ++cand) {
       const int tpc = (tiles + cand - 1) / cand;
       const int chunks = (tiles + tpc - 1) / tpc;
       const int waves = (chunks * per_chunk_items + ctx->sm_count - 1) / ctx->sm_count;

@@ -531,11 +531,11 @@ def run_ours(args):
     for name, key in (("stats", "stats_bytes"), ("sweep", "sweep_bytes"), ("reduce", "reduce_bytes")):
         if name in per_class:
             gbs = sum(work[key]) / (per_class[name]["ms_per_step"] * 1e-3) / 1e9
-            launches = max(per_class[name]["launches_per_step"], 1.0)
+            class_launches = max(per_class[name]["launches_per_step"], 1.0)
             extra[name] = {"GB/s": gbs, "frac_of_copy_peak": gbs / pk["hbm_gbs"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
                            "algorithmic_bytes_per_layer": sum(work[key]) / L,
                            "us_per_layer": 1e3 * per_class[name]["ms_per_step"] / L,
-                           "launches_per_layer": launches / L,
+                           "launches_per_layer": class_launches / L,
                            "traffic": kernel_traffic(name, wl.name),
                            "traffic_unit": "dram bytes per layer's main launch (ncu, 2-layer capture of the same config)"}
     # the two phase-A sweeps evaluate one exp2 per logit on the special-function units: 16 per clock per SM

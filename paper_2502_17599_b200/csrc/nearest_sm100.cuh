@@ -358,6 +358,7 @@ nearest_kernel(const __grid_constant__ CUtensorMap map_kc, const NearestParams p
   // ------------------------------------------------------------------ common exit
   tc_fence_before_sync();
   __syncthreads();
+  drain_after_abort(abort_flag);
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kNtTmemCols);

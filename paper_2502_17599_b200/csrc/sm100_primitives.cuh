@@ -72,6 +72,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return true;
 }
 
+// Exit path of a pipeline whose wait ran out: copies and UMMAs already issued cannot be recalled and may still be
+// writing this block's shared or tensor memory.  Nothing can wait for them by name any more (the barrier protocol
+// is broken by then), so the block idles for a bounded time, far longer than any single copy or instruction takes,
+// before it releases its tensor memory and returns.
+__device__ __forceinline__ void drain_after_abort(volatile int* abort_flag) {
+  if (*abort_flag == 0) return;
+  const long long t0 = clock64();
+  while (clock64() - t0 < 200000ll) __nanosleep(1000);
+}
+
 // ---- TMA ---------------------------------------------------------------------------------------
 // 3-D tiled load global -> shared, completion counted in bytes on `bar`.  The innermost coordinate
 // times the element size must be a multiple of 16 bytes (all callers pass multiples of 64 bf16).

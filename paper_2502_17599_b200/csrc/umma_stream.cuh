@@ -233,6 +233,7 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   // ------------------------------------------------------------------ common exit
   tc_fence_before_sync();
   __syncthreads();
+  drain_after_abort(abort_flag);
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kUsTmemCols);

@@ -471,6 +471,7 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
   // ------------------------------------------------------------------ common exit
   tc_fence_before_sync();
   __syncthreads();
+  drain_after_abort(abort_flag);
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kWsTmemCols);

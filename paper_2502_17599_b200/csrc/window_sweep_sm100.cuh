@@ -391,6 +391,7 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
   // ------------------------------------------------------------------ common exit
   tc_fence_before_sync();
   __syncthreads();
+  drain_after_abort(abort_flag);
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kSwTmemCols);

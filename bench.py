@@ -279,10 +279,10 @@ def algorithmic_work(wl, budgets):
 CSRC = "paper_2502_17599_b200/csrc/"
 KERNEL_TRAFFIC = {
     # class: (bytes per launch, source files, sha256[:16] of their concatenation)
-    "nearest": (140.1e6, (CSRC + "nearest_sm100.cuh", CSRC + "sm100_primitives.cuh"), None),
-    "stats": (None, (CSRC + "window_stats_sm100.cuh", CSRC + "sm100_primitives.cuh"), None),
-    "sweep": (None, (CSRC + "window_sweep_sm100.cuh", CSRC + "sm100_primitives.cuh"), None),
-    "reduce": (None, (CSRC + "group_reduce.cuh",), None),
+    "nearest": (138.9e6, (CSRC + "nearest_sm100.cuh", CSRC + "sm100_primitives.cuh"), "802a52cd62a33938"),
+    "stats": (136.8e6, (CSRC + "window_stats_sm100.cuh", CSRC + "sm100_primitives.cuh"), "8796929e3a0b9995"),
+    "sweep": (137.3e6, (CSRC + "window_sweep_sm100.cuh", CSRC + "sm100_primitives.cuh"), "73e64b1d83362859"),
+    "reduce": (288.1e6, (CSRC + "group_reduce.cuh",), "71af809bda69dc5b"),
 }
 NOMINAL_HBM_GBS = 8000.0     # the nominal figure the target is worded against; the measured copy peak is the denominator of `frac`
 

@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--no-prompt-scores", action="store_true",
                     help="skip the context measurement of Eq. 8 taken over every prompt row (one layer)")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--oracle-sampled", action="store_true",
+                    help="time the oracle on the bounded sample even where the whole pass would be small enough")
     ap.add_argument("--oracle-whole-pass", action="store_true",
                     help="time the oracle on the whole pass, un-sampled, whatever its size (minutes for the large workloads)")
     return ap.parse_args()
@@ -87,7 +89,7 @@ def oracle_whole_pass_seconds(wl):
     return time.perf_counter() - t0, "whole pass, every layer and head, un-sampled"
 
 
-def oracle_sample_seconds(wl, budgets=None, whole_pass=False):
+def oracle_sample_seconds(wl, budgets=None, whole_pass=False, sampled=False):
     """Times the oracle, as it stands, on a bounded sample of the workload and scales it to the whole pass.
 
     `budgets`: the (S, M, N) rows of the measured run (read back from the device), so that the sample has a
@@ -105,7 +107,7 @@ def oracle_sample_seconds(wl, budgets=None, whole_pass=False):
     real = budgets is not None
     rows = [tuple(int(x) for x in b) for b in budgets] if real else uniform_budgets(wl)
     n = wl.n_tokens
-    if whole_pass or (similarity_entries(wl, rows) <= WHOLE_PASS_MAX_SIMILARITIES and wl.n_layers * n <= 1.2e6):
+    if whole_pass or (not sampled and similarity_entries(wl, rows) <= WHOLE_PASS_MAX_SIMILARITIES and wl.n_layers * n <= 1.2e6):
         sec, desc = oracle_whole_pass_seconds(wl)
         return sec, desc, False
     work = [(n - s) * s for s, _, _ in rows]
@@ -167,7 +169,7 @@ def run_reference(args):
     times = []
     desc, extrapolated = "", False
     for i in range(args.warmup + args.steps):
-        dt, desc, extrapolated = oracle_sample_seconds(wl, whole_pass=args.oracle_whole_pass)
+        dt, desc, extrapolated = oracle_sample_seconds(wl, whole_pass=args.oracle_whole_pass, sampled=args.oracle_sampled)
         if i >= args.warmup:
             times.append(dt)
     sec = sum(times) / len(times)
@@ -556,7 +558,8 @@ def run_ours(args):
 
     cpu = None
     if not args.no_cpu_baseline:
-        sec, desc, extrapolated = oracle_sample_seconds(wl, cp.budgets.cpu().numpy(), whole_pass=args.oracle_whole_pass)
+        sec, desc, extrapolated = oracle_sample_seconds(wl, cp.budgets.cpu().numpy(), whole_pass=args.oracle_whole_pass,
+                                                           sampled=args.oracle_sampled)
         cpu = {"value": oracle_throughput(wl, sec), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                "sample": desc, "pass_seconds": sec, "extrapolated": extrapolated}
 

@@ -28,6 +28,11 @@ def small_cases():
         # shapes that take the tensor-core phase-A kernels (bf16, d=128, window 32 or 64)
         W.small_variant("tc_w32", window=32, seed=4),
         W.small_variant("tc_w64_wide", window=64, n_q_heads=10, n_kv_heads=2, seed=5),   # 320 query rows per KV group
+        # grouped-query shapes that take the grouped scores sweep (129 .. 256 query rows per KV head, window 32):
+        # 160 rows with a ragged last key block of one tile, and the full 256 rows (fewer key stages fit)
+        W.small_variant("tc_w32_g5", window=32, n_q_heads=10, n_kv_heads=2, seed=6,
+                        spans=((0, 37, 0), (37, 37 + 9 * 61, 1), (37 + 9 * 61, 37 + 9 * 61 + 40, 0))),   # n = 626 = 2 x 256 + 114
+        W.small_variant("tc_w32_g8", window=32, n_q_heads=16, n_kv_heads=2, seed=7),
         W.WORKLOADS["long_video_19k"].with_(name="long_video_19k_2l", n_layers=2),
     ]
 

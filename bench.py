@@ -44,6 +44,10 @@ def parse_args():
     ap.add_argument("--no-prompt-scores", action="store_true",
                     help="skip the context measurement of Eq. 8 taken over every prompt row (one layer)")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--shard", default="prompts", choices=["prompts", "layers"],
+                    help="with --gpus N > 1: every rank its own prompt (weak scaling, no collective; the default), or ONE "
+                         "prompt with its layers dealt round-robin to the ranks and one all-reduce of the L entropies "
+                         "between the phases (strong scaling)")
     ap.add_argument("--oracle-sampled", action="store_true",
                     help="time the oracle on the bounded sample even where the whole pass would be small enough")
     ap.add_argument("--oracle-whole-pass", action="store_true",
@@ -348,13 +352,19 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
 
-    wl = rank_workload(args.workload, rank, args.layers)
+    by_layer = args.shard == "layers" and world > 1
+    wl = rank_workload(args.workload, 0 if by_layer else rank, args.layers)
     L = wl.n_layers
+    shard = (rank, world) if by_layer else None
+    from paper_2502_17599_b200.pipeline import owned_layers
+    mine = set(owned_layers(L, rank, world)) if by_layer else set(range(L))
     qs, ks, vs = [], [], []
     for l in range(L):
-        q, k, v = W.make_layer(wl, l, "cuda")
+        q, k, v = W.make_layer(wl, l, "cuda") if l in mine else (None, None, None)
         qs.append(q); ks.append(k); vs.append(v)
-    input_bytes = sum(t.numel() * t.element_size() for ts in (qs, ks, vs) for t in ts)
+    if by_layer:      # the legs below walk every layer of the prompt on one GPU
+        args.eager = args.no_e2e = args.no_decode = args.no_prompt_scores = True
+    input_bytes = sum(t.numel() * t.element_size() for ts in (qs, ks, vs) for t in ts if t is not None)
     cp = CompressionPass(wl, n_streams=args.streams)
     stream = torch.cuda.current_stream()
 
@@ -368,7 +378,7 @@ def run_ours(args):
     # single launch on the host.  Kernel-level times come from a second region of the same K steps
     # run eagerly with every launch bracketed by events, whose overhead must not be in the headline.
     kernels_per_pass = cp.capture(qs, ks, vs) if not args.eager else None
-    step = cp.replay if not args.eager else (lambda: cp.run(qs, ks, vs))
+    step = cp.replay if not args.eager else (lambda: cp.run(qs, ks, vs, layer_shard=shard))
     for _ in range(args.warmup):
         step()
     cp.check()
@@ -392,7 +402,7 @@ def run_ours(args):
     cp.ctx.profile_enable(True)
     barrier()
     for _ in range(args.steps):
-        cp.run(qs, ks, vs, single_stream=True)      # one stream: a launch's events bracket that launch alone
+        cp.run(qs, ks, vs, single_stream=True, layer_shard=shard)      # one stream: a launch's events bracket that launch alone
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     dropped = cp.ctx.profile_dropped()
@@ -403,7 +413,7 @@ def run_ours(args):
         raise RuntimeError(f"{dropped} launches of the per-kernel timing region went untimed (event pool full): "
                            "per-class times would not cover --steps steps; use fewer steps")
     ms_step = max_over_ranks(ms_total, world, "cuda") / args.steps
-    value = whole_job_throughput(wl, world, ms_step)
+    value = whole_job_throughput(wl, 1 if by_layer else world, ms_step)      # one prompt in all when sharded by layer
 
     # context: one decoding step's attention (Eq. 3) over all layers, compressed caches against full ones
     decode = None
@@ -500,7 +510,9 @@ def run_ours(args):
         return
 
     pk = peaks()
-    work = algorithmic_work(wl, budgets)
+    own = sorted(mine)
+    L_local = len(own)
+    work = algorithmic_work(wl, budgets[own])          # rank 0's kernel times cover its own layers
     per_class = {name: {"ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps}
                  for name, (ms, cnt) in prof.items() if cnt}
     total_prof = sum(v["ms_per_step"] for v in per_class.values()) or 1.0
@@ -535,13 +547,13 @@ def run_ours(args):
             gbs = sum(work[key]) / (per_class[name]["ms_per_step"] * 1e-3) / 1e9
             class_launches = max(per_class[name]["launches_per_step"], 1.0)
             extra[name] = {"GB/s": gbs, "frac_of_copy_peak": gbs / pk["hbm_gbs"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-                           "algorithmic_bytes_per_layer": sum(work[key]) / L,
-                           "us_per_layer": 1e3 * per_class[name]["ms_per_step"] / L,
-                           "launches_per_layer": class_launches / L,
+                           "algorithmic_bytes_per_layer": sum(work[key]) / L_local,
+                           "us_per_layer": 1e3 * per_class[name]["ms_per_step"] / L_local,
+                           "launches_per_layer": class_launches / L_local,
                            "traffic": kernel_traffic(name, wl.name),
                            "traffic_unit": "dram bytes per layer's main launch (ncu, 2-layer capture of the same config)"}
     # the two phase-A sweeps evaluate one exp2 per logit on the special-function units: 16 per clock per SM
-    exps = float(L) * wl.n_q_heads * wl.window * wl.n_tokens
+    exps = float(L_local) * wl.n_q_heads * wl.window * wl.n_tokens
     sfu_peak = 148 * 16 * (clocks["sm_max_mhz"] or 1965.0) * 1e6 if clocks else None
     for name in ("stats", "sweep"):
         if name in per_class and sfu_peak:
@@ -565,11 +577,12 @@ def run_ours(args):
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong" if by_layer else "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": wl.name, "shape": wl.description, "global_budget": wl.global_budget,
                    "input_bytes": input_bytes, "l2": "inputs larger than L2 (no flush needed)" if input_bytes > 256e6 else "inputs fit L2",
-                   "parallelism": f"independent prompts x{world}",
+                   "parallelism": (f"one prompt, layers round-robin over {world} ranks, one all-reduce of {L} entropies"
+                                   if by_layer else f"independent prompts x{world}"),
                    "launch": ("eager launches" if args.eager else f"one CUDA-graph replay per step ({kernels_per_pass} kernels)")
                              + f", layers alternate between {len(cp.contexts)} streams"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),

@@ -9,6 +9,21 @@ from . import binding
 from .workloads import Workload
 
 
+def owned_layers(n_layers: int, rank: int, world: int) -> list[int]:
+    """Layers rank `rank` of `world` processes when ONE prompt is sharded by layer: round-robin, so that the
+    layers a model's depth makes expensive (large budgets cluster) spread over the ranks."""
+    return [l for l in range(n_layers) if l % world == rank]
+
+
+def exchange_entropies(entropy: torch.Tensor, group=None) -> None:
+    """The one exchange step of a layer-sharded pass (Eq. 7's softmax runs over ALL layers): `entropy` holds
+    this rank's layers and zeros elsewhere; after the call every rank holds every layer's value (a sum over
+    disjoint supports, so the result is exact and the same bits on every rank).  L floats: latency only."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(entropy, op=dist.ReduceOp.SUM, group=group)
+
+
 class CompressionPass:
     """Buffers and call sequence of one prompt's pass on one GPU.
 
@@ -66,7 +81,7 @@ class CompressionPass:
             main.wait_event(ev)
 
     def run(self, q_layers, k_layers, v_layers, stream=None, single_stream=False, qk_ready=None, v_ready=None,
-            budgets_done=None, layer_done=None, max_lanes=None):
+            budgets_done=None, layer_done=None, max_lanes=None, layer_shard=None, exchange=None):
         """Enqueues the whole pass.  Inputs are lists of per-layer device tensors; results stay on the
         device in this object's buffers.  The work is ordered after what `stream` (default: torch's
         current stream) holds and `stream` waits for all of it.  With `single_stream` everything goes to
@@ -75,8 +90,14 @@ class CompressionPass:
         place (copies still in flight on another stream): phase A of a layer waits for the first,
         phase B for the second.  `budgets_done` (an event) is recorded once the budgets are written,
         `layer_done[l]` (events) once layer l's compressed cache is: a caller can start copying results
-        out while later layers are still being compressed.  `max_lanes` limits the streams used."""
+        out while later layers are still being compressed.  `max_lanes` limits the streams used.
+        `layer_shard=(rank, world)`: this process runs only the layers `owned_layers` deals it (the other
+        entries of the input lists are not read and may be None); the L entropies are exchanged between the
+        two phases, so every rank computes the same budgets, and each rank's outputs hold its own layers
+        only.  `exchange` replaces the collective (a callable taking the entropy tensor; used to emulate the
+        other ranks on one GPU)."""
         L = self.wl.n_layers
+        mine = list(range(L)) if layer_shard is None else owned_layers(L, *layer_shard)
         main = stream if stream is not None else torch.cuda.current_stream()
         if single_stream or not self.streams:
             lanes = [(self.contexts[0], main, self.row_stats[0])]
@@ -85,20 +106,28 @@ class CompressionPass:
             if max_lanes is not None:
                 lanes = lanes[: max(1, max_lanes)]
             self._fork(main)
-        for l in range(L):
-            c, s, rs = lanes[l % len(lanes)]
+        if layer_shard is not None:
+            with torch.cuda.stream(main):
+                self.entropy.zero_()                  # the other ranks' layers must read as zero in the exchange
+            if len(lanes) > 1:
+                self._fork(main)
+        for i, l in enumerate(mine):
+            c, s, rs = lanes[i % len(lanes)]
             if qk_ready is not None:
                 s.wait_event(qk_ready[l])
             c.window_scores(l, q_layers[l], k_layers[l], rs, self.scores[l], self.entropy, s)
         if len(lanes) > 1:
             self._join(main)
+        if layer_shard is not None:
+            with torch.cuda.stream(main):
+                (exchange or exchange_entropies)(self.entropy)
         self.ctx.allocate_budgets(self.entropy, self.budgets, main)      # Eq. 7 needs every layer's entropy
         if budgets_done is not None:
             budgets_done.record(main)
         if len(lanes) > 1:
             self._fork(main)
-        for l in range(L):
-            c, s, _ = lanes[l % len(lanes)]
+        for i, l in enumerate(mine):
+            c, s, _ = lanes[i % len(lanes)]
             if v_ready is not None:
                 s.wait_event(v_ready[l])
             c.compress_layer(l, k_layers[l], v_layers[l], self.scores[l], self.budgets, self.k_out[l], self.v_out[l],

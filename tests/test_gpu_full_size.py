@@ -206,3 +206,39 @@ def test_full_size_variants_ablation_modes_vision_to_text_term_and_decoding_step
     want_out = O.decode_attention(P.np64(q_new), P.np64(cp.k_out[layer, :, :S]), P.np64(cp.v_out[layer, :, :S]))
     np.testing.assert_allclose(P.np64(out), want_out, rtol=1e-4, atol=1e-4)
     cp.close()
+
+
+def test_one_prompt_sharded_by_layer_gives_the_unsharded_results():
+    """The layer-sharded pass (one prompt, layers dealt round-robin to ranks, entropies exchanged between the
+    phases) emulated on one GPU: two shards run one after the other, each receiving the other's entropies through
+    the exchange hook.  Budgets and every owned layer's outputs equal the unsharded pass bit for bit."""
+    from paper_2502_17599_b200.pipeline import CompressionPass, owned_layers
+    wl = W.WORKLOADS["long_video_19k"].with_(name="long_video_19k_6l", n_layers=6)
+    L = wl.n_layers
+    qs, ks, vs = [], [], []
+    for l in range(L):
+        q, k, v = W.make_layer(wl, l, "cuda")
+        qs.append(q); ks.append(k); vs.append(v)
+    whole = CompressionPass(wl, n_streams=2)
+    whole.run(qs, ks, vs)
+    whole.check()
+    for rank in range(2):
+        mine = owned_layers(L, rank, 2)
+        others = torch.zeros_like(whole.entropy)
+        for l in range(L):
+            if l not in mine:
+                others[l] = whole.entropy[l]
+        part = CompressionPass(wl, n_streams=2)
+        part.run([q if l in mine else None for l, q in enumerate(qs)], ks, vs, layer_shard=(rank, 2),
+                 exchange=lambda e: e.add_(others))
+        part.check()
+        assert torch.equal(part.entropy, whole.entropy) and torch.equal(part.budgets, whole.budgets)
+        for l in mine:
+            S = int(whole.budgets[l, 0])
+            assert torch.equal(part.scores[l], whole.scores[l])
+            assert torch.equal(part.idx_c[l, :, :S], whole.idx_c[l, :, :S])
+            assert torch.equal(part.counts[l, :, :S], whole.counts[l, :, :S])
+            assert torch.equal(part.k_out[l, :, :S], whole.k_out[l, :, :S])
+            assert torch.equal(part.v_out[l, :, :S], whole.v_out[l, :, :S])
+        part.close()
+    whole.close()

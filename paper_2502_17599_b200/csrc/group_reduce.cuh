@@ -6,7 +6,9 @@
 // less-important rows (their target slot, their row), so after the sort every slot's rows are
 // contiguous, the kept row first, then its members in ascending token order (stability).  Warps then
 // walk fixed 128-row chunks of the sorted list, summing in fp32 in list order: no row needs a
-// look-up of its own, every load address comes from the list.  A slot whose rows lie inside one chunk
+// look-up of its own, every load address comes from the list (32 entries per coalesced load, handed
+// round by shuffle; batches of 8 rows inside one slot's segment are added without a branch, two
+// batches in flight).  A slot whose rows lie inside one chunk
 // is finished on the spot (one division, one rounding), pieces of slots that cross chunk borders are
 // parked as partial sums and added up in chunk order by a second small kernel.
 // No floating-point atomics anywhere: two runs give identical bits.
@@ -238,6 +240,67 @@ __device__ __forceinline__ void store_row(T* p, int lane, const float (&x)[E], f
   for (int e = 0; e < E; ++e) p[lane * E + e] = from_f32<T>(x[e] / count);
 }
 
+// A lane's share of a row as loaded (E elements, not yet widened), and its addition to fp32 sums.
+template <typename T, int E> struct RawRow;
+template <> struct RawRow<__nv_bfloat16, 2> { uint32_t u; };
+template <> struct RawRow<__nv_bfloat16, 4> { uint2 u; };
+template <> struct RawRow<__nv_bfloat16, 8> { uint4 u; };
+template <int E> struct RawRow<float, E> { float f[E]; };
+
+__device__ __forceinline__ void add_bf16x2(float& lo, float& hi, uint32_t u) {
+  lo += __uint_as_float(u << 16);
+  hi += __uint_as_float(u & 0xffff0000u);
+}
+__device__ __forceinline__ void raw_load(RawRow<__nv_bfloat16, 2>& r, const char* p) { r.u = *reinterpret_cast<const uint32_t*>(p); }
+__device__ __forceinline__ void raw_load(RawRow<__nv_bfloat16, 4>& r, const char* p) { r.u = *reinterpret_cast<const uint2*>(p); }
+__device__ __forceinline__ void raw_load(RawRow<__nv_bfloat16, 8>& r, const char* p) { r.u = *reinterpret_cast<const uint4*>(p); }
+template <int E>
+__device__ __forceinline__ void raw_load(RawRow<float, E>& r, const char* p) {
+#pragma unroll
+  for (int e = 0; e < E; ++e) r.f[e] = reinterpret_cast<const float*>(p)[e];
+}
+__device__ __forceinline__ void raw_add(float (&a)[2], const RawRow<__nv_bfloat16, 2>& r) { add_bf16x2(a[0], a[1], r.u); }
+__device__ __forceinline__ void raw_add(float (&a)[4], const RawRow<__nv_bfloat16, 4>& r) {
+  add_bf16x2(a[0], a[1], r.u.x);
+  add_bf16x2(a[2], a[3], r.u.y);
+}
+__device__ __forceinline__ void raw_add(float (&a)[8], const RawRow<__nv_bfloat16, 8>& r) {
+  add_bf16x2(a[0], a[1], r.u.x);
+  add_bf16x2(a[2], a[3], r.u.y);
+  add_bf16x2(a[4], a[5], r.u.z);
+  add_bf16x2(a[6], a[7], r.u.w);
+}
+template <int E>
+__device__ __forceinline__ void raw_add(float (&a)[E], const RawRow<float, E>& r) {
+#pragma unroll
+  for (int e = 0; e < E; ++e) a[e] += r.f[e];
+}
+
+template <int E> struct SegSums { float a[E]; };
+
+// End of a piece of a slot's segment inside a chunk.  A segment that starts and ends in the chunk is finished here
+// (one division, one rounding; a slot without members keeps its row as it is); a piece of a segment that crosses
+// the chunk's border is parked for seg_border_kernel.  The walker calls this from rolled loops only, so that it
+// holds few copies of this code: with one copy per row of an unrolled batch it outgrew the instruction cache and
+// ran at half speed wherever most slots have no members (a call out of line was slower too: the batches in
+// flight had to be saved around it).
+template <typename T, int E>
+__device__ __forceinline__ void seg_end_piece(SegSums<E> sums, int members, bool whole, T* out_row, float* park_row,
+                                           int32_t* count_out, int lane) {
+  if (whole) {
+    if (members == 1) {
+#pragma unroll
+      for (int e = 0; e < E; ++e) out_row[lane * E + e] = from_f32<T>(sums.a[e]);
+    } else {
+      store_row<T, E>(out_row, lane, sums.a, (float)members);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < E; ++e) park_row[lane * E + e] = sums.a[e];
+  }
+  if (count_out != nullptr) *count_out = members;
+}
+
 // grid = (chunks / kSegWarps, heads, 2): blockIdx.z picks the tensor (0 keys, 1 values), so that twice
 // as many warps keep rows in flight; the z = 0 warps also record segment bounds and counts.  Every slot
 // has at least one row in the list (its kept row), so every slot's bounds get written.
@@ -252,85 +315,109 @@ seg_reduce_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_
   const int g = blockIdx.y, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int tensor = blockIdx.z;
   const bool book = tensor == 0 && lane == 0;            // the one lane that writes bounds and counts
-  const int chunk = blockIdx.x * kSegWarps + warp;
+  // The list's last chunks first: slots are in token order, so the recent window's slots (most of them without
+  // members: one segment per row, the slowest chunks) come last in the list and would otherwise form the tail.
+  const int chunk = n_chunks - 1 - ((int)blockIdx.x * kSegWarps + warp);
   const int S = min(budget_row[0], cap);
   const int q0 = chunk * kSegChunk;
-  if (S <= 0 || q0 >= n) return;
+  if (S <= 0 || chunk < 0 || q0 >= n) return;
   const int q1 = min(q0 + kSegChunk, n);
   // the grouped list is in the buffer the last executed sort pass wrote: pass p writes buffer p % 2
   const bool in_b = ((sort_passes_done(S, max_passes) - 1) & 1) != 0;
   const int32_t* kg = (in_b ? keys_b : keys_a) + (size_t)g * n;
   const int32_t* rg = (in_b ? rows_b : rows_a) + (size_t)g * n;
-  const T* x_g = (tensor == 0 ? k : v) + (size_t)g * n * D;
+  const char* x_bytes = reinterpret_cast<const char*>((tensor == 0 ? k : v) + (size_t)g * n * D) + lane * (E * sizeof(T));
   T* out_g = (tensor == 0 ? k_out : v_out) + (size_t)g * cap * D;
   int32_t* st = seg_start + (size_t)g * n;
   int32_t* en = seg_end + (size_t)g * n;
 
-  float acc[E];
-  int members = 0;
+  SegSums<E> acc;
+  int members = 0;                  // rows of the slot summed so far, the kept row included
   int cur = min(max(kg[q0], 0), S - 1);
   bool started_here = (q0 == 0) || (kg[q0 - 1] != kg[q0]);
 
-  // `members` counts the rows of the slot summed so far, the kept row included
   auto begin_segment = [&](int slot, bool fresh, int q) {
     members = 0;
 #pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    for (int e = 0; e < E; ++e) acc.a[e] = 0.f;
     if (fresh && book) st[slot] = q;
   };
   auto end_piece = [&](int slot, bool fresh, bool ended, int q_end) {
     if (ended && book) en[slot] = q_end;
-    if (fresh && ended) {
-      store_row<T, E>(out_g + (size_t)slot * D, lane, acc, (float)members);
-      if (book) counts[(size_t)g * cap + slot] = members;
-    } else {
-      const int which = fresh ? 1 : 0;
-      float* cp = carry_ptr<D>(carry, g, chunk, which, n_chunks) + tensor * D;
-#pragma unroll
-      for (int e = 0; e < E; ++e) cp[lane * E + e] = acc[e];
-      if (book) carry_cnt[((size_t)g * n_chunks + chunk) * 2 + which] = members;
-    }
+    const bool whole = fresh && ended;
+    const int which = fresh ? 1 : 0;
+    int32_t* count_out = !book ? nullptr
+                         : whole ? counts + (size_t)g * cap + slot
+                                 : carry_cnt + ((size_t)g * n_chunks + chunk) * 2 + which;
+    seg_end_piece<T, E>(acc, members, whole, out_g + (size_t)slot * D,
+                        carry_ptr<D>(carry, g, chunk, which, n_chunks) + tensor * D, count_out, lane);
   };
 
   begin_segment(cur, started_here, q0);
-  constexpr int kBatch = 32 / E;                    // 32 row elements per lane in flight
-  // the (slot, row) pairs of the next batch are fetched while the rows of this one are in flight
-  int key[kBatch], row[kBatch];
-#pragma unroll
-  for (int b = 0; b < kBatch; ++b) {
-    const int q = min(q0 + b, q1 - 1);
-    key[b] = kg[q];
-    row[b] = rg[q];
+  // Rounds of 32 list entries: lane l holds entry qb + l (one coalesced load per array and round, the next round's
+  // in flight during this one) and the entries reach the other lanes by shuffle.  A round is cut into batches of
+  // 8 rows (fewer for wide rows), two batches in flight.  A batch that lies inside the current slot's segment (the common case wherever slots
+  // have many members) is summed without a branch; the others go row by row.
+  using Raw = RawRow<T, E>;
+  constexpr int kBatch = sizeof(Raw) <= 8 ? 8 : (sizeof(Raw) <= 16 ? 4 : 2);      // two batches of 64 bytes per lane in flight
+  int key_l, row_l;
+  {
+    const int q = min(q0 + lane, q1 - 1);
+    key_l = kg[q];
+    row_l = rg[q];
   }
-  for (int qb = q0; qb < q1; qb += kBatch) {
-    float x[kBatch][E];
-    int key_now[kBatch];
-#pragma unroll
-    for (int b = 0; b < kBatch; ++b) {
-      key_now[b] = min(max(key[b], 0), S - 1);
-      load_row<T, E>(x_g + (size_t)min(max(row[b], 0), n - 1) * D, lane, x[b]);
+#pragma unroll 1
+  for (int qb = q0; qb < q1; qb += 32) {
+    const int key_r = min(max(key_l, 0), S - 1);
+    const uint32_t off_r = (uint32_t)min(max(row_l, 0), n - 1) * (uint32_t)(D * sizeof(T));
+    const bool live = qb + lane < q1;
+    if (qb + 32 < q1) {
+      const int q = min(qb + 32 + lane, q1 - 1);
+      key_l = kg[q];
+      row_l = rg[q];
     }
-    if (qb + kBatch < q1) {
+    auto fetch = [&](Raw (&x)[kBatch], int b0) {
 #pragma unroll
-      for (int b = 0; b < kBatch; ++b) {
-        const int q = min(qb + kBatch + b, q1 - 1);
-        key[b] = kg[q];
-        row[b] = rg[q];
-      }
-    }
+      for (int b = 0; b < kBatch; ++b) raw_load(x[b], x_bytes + __shfl_sync(0xffffffffu, off_r, b0 + b));
+    };
+    auto consume = [&](const Raw (&x)[kBatch], int b0) {
+      const unsigned int brk = (__ballot_sync(0xffffffffu, !live || key_r != cur) >> b0) & ((1u << kBatch) - 1u);
+      if (brk == 0u) {
 #pragma unroll
-    for (int b = 0; b < kBatch; ++b) {
-      if (qb + b < q1) {
-        if (key_now[b] != cur) {
-          end_piece(cur, started_here, true, qb + b);
-          cur = key_now[b];
-          started_here = true;
-          begin_segment(cur, true, qb + b);
+        for (int b = 0; b < kBatch; ++b) raw_add(acc.a, x[b]);
+        members += kBatch;
+      } else {
+        // row by row, one copy of the code: the rows are read again (they are in the first-level cache, the
+        // batch's loads brought them), the next row's load in flight while this row is handled
+        Raw nxt;
+        raw_load(nxt, x_bytes + __shfl_sync(0xffffffffu, off_r, b0));
+#pragma unroll 1
+        for (int b = 0; b < kBatch; ++b) {
+          const Raw now = nxt;
+          raw_load(nxt, x_bytes + __shfl_sync(0xffffffffu, off_r, min(b0 + b + 1, 31)));
+          const int key_b = __shfl_sync(0xffffffffu, key_r, b0 + b);
+          if (qb + b0 + b < q1) {
+            if (key_b != cur) {
+              end_piece(cur, started_here, true, qb + b0 + b);
+              cur = key_b;
+              started_here = true;
+              begin_segment(cur, true, qb + b0 + b);
+            }
+            raw_add(acc.a, now);
+            ++members;
+          }
         }
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[e] += x[b][e];
-        ++members;
       }
+    };
+    // entries past the chunk's end repeat its last entry: their loads are in bounds and their rows are not added
+    Raw xa[kBatch], xb[kBatch];
+    fetch(xa, 0);
+#pragma unroll 1
+    for (int h = 0; h < 32; h += 2 * kBatch) {
+      fetch(xb, h + kBatch);
+      consume(xa, h);
+      if (h + 2 * kBatch < 32) fetch(xa, h + 2 * kBatch);
+      consume(xb, h + kBatch);
     }
   }
   const bool ended = (q1 == n) || (min(max(kg[q1], 0), S - 1) != cur);

@@ -207,8 +207,20 @@ struct StatsPolicy {
 // p_vis / Hq, and e * vis.y is the full-softmax probability; for a text key exp2(t - text.x) * text.y
 // is the full-softmax probability.  A row that sees no visual key gets (+huge, 0): e = 0.
 // ---------------------------------------------------------------------------------------------
+// Two layouts of the tables: (ref, ratio) per column, or, for the sweep that works on pairs of columns with
+// packed arithmetic, four floats per pair of columns: (-ref, -ref', ratio, ratio').
+__device__ __forceinline__ void store_sweep_coef(float2* table, size_t col, float2 c, bool paired) {
+  if (!paired) {
+    table[col] = c;
+  } else {
+    float* f = reinterpret_cast<float*>(table) + (col / 2) * 4 + (col & 1);
+    f[0] = -c.x;
+    f[2] = c.y;
+  }
+}
+
 __global__ void sweep_coef_kernel(const float* __restrict__ row_stats, float2* __restrict__ vis,
-                                  float2* __restrict__ text, int rows, float hq) {
+                                  float2* __restrict__ text, int rows, float hq, bool paired) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= rows) return;
   const float4 s = reinterpret_cast<const float4*>(row_stats)[c];
@@ -217,8 +229,8 @@ __global__ void sweep_coef_kernel(const float* __restrict__ row_stats, float2* _
     a.x = fmaf(s.z, kLog2e, log2f(s.w * hq));
     a.y = hq * s.w * expf(s.z - s.x) / s.y;
   }
-  vis[c] = a;
-  text[c] = make_float2(s.x * kLog2e, 1.f / s.y);
+  store_sweep_coef(vis, c, a, paired);
+  store_sweep_coef(text, c, make_float2(s.x * kLog2e, 1.f / s.y), paired);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -226,6 +226,7 @@ meda_status launch_stats_fast(meda_ctx* ctx, const void* q_win, const void* k, f
   prm.row_stats = row_stats;
   prm.coef_vis = ctx->ws.coef_vis;
   prm.coef_text = ctx->ws.coef_text;
+  prm.coef_paired = ctx->fast_sweep_grouped ? 1 : 0;
   prm.counters = ctx->ws.stats_counters;
   prm.n = c.n_tokens; prm.hq = c.n_q_heads; prm.group = ctx->group; prm.w = c.window;
   prm.cols = ctx->group * c.window;
@@ -315,7 +316,7 @@ meda_status launch_sweep_fast(meda_ctx* ctx, int32_t layer, const void* q_win, c
   if (!coef_ready) {
     LaunchScope scope(ctx, MEDA_K_STATS_COMBINE, st);
     sweep_coef_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_stats, ctx->ws.coef_vis, ctx->ws.coef_text, rows,
-                                                          (float)c.n_q_heads);
+                                                          (float)c.n_q_heads, grouped);
   }
   if (grouped) {
     LaunchScope scope(ctx, MEDA_K_SWEEP, st);

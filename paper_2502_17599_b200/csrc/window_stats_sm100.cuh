@@ -51,6 +51,7 @@ struct WinStatsParams {
   float* row_stats;              // [Hq][w][4]  (written by the merging warps)
   float2* coef_vis;              // [Hq * w]    per-column constants of the second sweep, or null
   float2* coef_text;             // [Hq * w]
+  int coef_paired;               // 0: (ref, ratio) per column; 1: (-ref, -ref', ratio, ratio') per pair of columns
   unsigned int* counters;        // [n_groups * row_blocks * 8], zero between launches
   int n, hq, group, w, cols;     // cols = group * w query rows per KV group
   int row_blocks;                // ceil(cols / 256)
@@ -234,8 +235,8 @@ __device__ __forceinline__ void win_stats_finish_row(const WinStatsParams& p, in
       a.x = fmaf(mv, kLog2e, log2f(zv * (float)p.hq));
       a.y = (float)p.hq * zv * expf(mv - m) / z;
     }
-    p.coef_vis[row] = a;
-    p.coef_text[row] = make_float2(m * kLog2e, 1.f / z);
+    store_sweep_coef(p.coef_vis, row, a, p.coef_paired != 0);
+    store_sweep_coef(p.coef_text, row, make_float2(m * kLog2e, 1.f / z), p.coef_paired != 0);
   }
 }
 

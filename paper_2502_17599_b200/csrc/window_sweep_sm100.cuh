@@ -17,9 +17,11 @@
 //    attention across the KV heads (Sum_i a_i ln a_i splits by row, so the four owners never have to meet)
 //    and a partial score; the four partial scores of a key are added through shared memory by the k = 0 warp.
 //  * One exponential per logit serves both softmaxes (the visual normaliser sits in the exponent's
-//    reference, see sweep_coef).  With a multiply-add before it, a multiply-add and an addition after it
-//    and half a shared-memory load per logit, the sweep is bound by the instructions it issues before the
-//    special-function unit saturates: no exponential is moved to the FMA pipes here.
+//    reference, see sweep_coef).  The arithmetic around it works on pairs of window rows with packed fp32
+//    instructions (the constants of a pair of columns are stored as one 16-byte entry whose halves are packed
+//    operands as they come out of shared memory): the sweep is bound by the instructions it issues before the
+//    special-function unit saturates, and for the same reason no exponential is moved to the FMA pipes here
+//    (a quarter of them as polynomials made the sweep 6 % slower, half of them 15 %).
 //  * The block that finishes last adds the entropy partials of all blocks in a fixed order.
 #pragma once
 
@@ -39,7 +41,7 @@ constexpr int kSwPartDepth = 4;                            // partial-score buff
 
 struct WinSweepParams {
   const uint8_t* modality;     // padded to a multiple of 256 (+128) with the value 2
-  const float2* vis;           // [Hq * w] per-column constants, see sweep_coef_kernel
+  const float2* vis;           // [Hq * w] per-column constants in the paired layout, see store_sweep_coef
   const float2* text;          // [Hq * w]
   const float* row_stats;      // [Hq][w][4] (the entropy's row count comes from it)
   float* scores;               // [Hkv][n] or null
@@ -225,10 +227,11 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     const int k = ewarp / 4;                      // quarter of the window rows this warp owns
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const int heads = p.cols / W;                 // query heads per KV head
-    float abar[2][R];                             // this thread's share of two keys' head-averaged attention
+    // this thread's share of two keys' head-averaged attention, as packed pairs of window rows
+    uint64_t abar[2][R / 2];
     float plogp = 0.f;                            // MODE 1
 #pragma unroll
-    for (int x = 0; x < R; ++x) abar[0][x] = abar[1][x] = 0.f;
+    for (int x = 0; x < R / 2; ++x) abar[0][x] = abar[1][x] = f32x2(0.f, 0.f);
     uint32_t b_cnt = 0, unit = 0;
     bool ok = true;
 
@@ -240,40 +243,46 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
       const int j = blk * 256 + T * 128 + key_in_tile;
       const bool valid = j < p.n;
       const int first_row = j - (p.n - W);                   // causal: window rows i >= first_row see key j
-      const bool masked = __any_sync(0xffffffffu, valid && first_row > k * R);
+      // keys past the prompt's end (zero rows of the last tile) take the masked path too: their exponentials are 0
+      const bool masked = __any_sync(0xffffffffu, !valid || first_row > k * R);
       bool good = mbar_wait(t_full + slot, tphase, abort_flag);
       good = __all_sync(0xffffffffu, good);
       if (!good) return false;
       tc_fence_after_sync();
       const uint32_t taddr = lane_addr + slot * 256u + (uint32_t)(k * R);
-      float score = 0.f;
       auto load = [&](uint32_t (&r)[R], int hl) {
         if constexpr (R == 8) tmem_ld_32x8_issue(taddr + (uint32_t)(hl * W), r);
         else tmem_ld_32x16_issue(taddr + (uint32_t)(hl * W), r);
       };
       // A text key takes the text constants and contributes nothing to the text-to-vision attention.
+      // The constants of a pair of columns are one 16-byte entry (-ref, -ref', ratio, ratio'): both halves are
+      // operands of packed fp32 instructions as they come out of shared memory.
       const float4* coef = (md == MEDA_VISUAL) ? cvis : ctext;
-      const float vflag = (valid && md == MEDA_VISUAL) ? 1.f : 0.f;
+      const float vf = (valid && md == MEDA_VISUAL) ? 1.f : 0.f;
+      const uint64_t vflag = f32x2(vf, vf), sc2x2 = f32x2(p.sc2, p.sc2);
+      uint64_t score2 = f32x2(0.f, 0.f);
       // The heads are software-pipelined by hand: the exponentials of head h are issued, then the sums of head
       // h - 1 (whose exponentials have completed meanwhile) are taken, then the columns of head h + 1 are fetched.
       // Issued in program order instead (exponentials, then their sums), every warp would stall on its own
       // special-function results with the unit idle behind it: the four warps of a scheduler leave a barrier
       // together and run in phase, so they cannot cover for each other.
       // The loop is unrolled to its maximum with a uniform branch per head: every offset is a constant.
+      // All sums are packed pairs (two window rows per instruction): the sweep is short of issue slots.
       uint32_t ra[R];
-      float e_prev[R], t_prev[MODE == 1 ? R : 1];
+      uint64_t e_prev[R / 2];
+      float t_prev[MODE == 1 ? R : 1];
       auto consume = [&](int c0) {                           // c0: pair index of the consumed head's first column
 #pragma unroll
-        for (int x = 0; x < R; x += 2) {
-          const float4 c = coef[c0 + x / 2];                  // read again rather than kept: registers are short
-          score = fmaf(e_prev[x], c.y, score);
-          score = fmaf(e_prev[x + 1], c.w, score);
+        for (int x = 0; x < R / 2; ++x) {
+          const float4 c = coef[c0 + x];                      // read again rather than kept: registers are short
+          score2 = fma_f32x2(e_prev[x], f32x2(c.z, c.w), score2);
           if (MODE == 0) {
-            abar[T][x] = fmaf(e_prev[x], vflag, abar[T][x]);
-            abar[T][x + 1] = fmaf(e_prev[x + 1], vflag, abar[T][x + 1]);
+            abar[T][x] = fma_f32x2(e_prev[x], vflag, abar[T][x]);
           } else {
-            plogp = fmaf(e_prev[x] * vflag, fmaf(t_prev[x], kLn2, p.ln_hq), plogp);
-            plogp = fmaf(e_prev[x + 1] * vflag, fmaf(t_prev[x + 1], kLn2, p.ln_hq), plogp);
+            float e0, e1;
+            f32x2_split(e_prev[x], e0, e1);
+            plogp = fmaf(e0 * vf, fmaf(t_prev[2 * x], kLn2, p.ln_hq), plogp);
+            plogp = fmaf(e1 * vf, fmaf(t_prev[2 * x + 1], kLn2, p.ln_hq), plogp);
           }
         }
       };
@@ -285,36 +294,39 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
           tmem_ld_pin_n<R>(ra);
           if (masked) {
 #pragma unroll
-            for (int x = 0; x < R; ++x) if (k * R + x < first_row) ra[x] = __float_as_uint(-1e30f);
+            for (int x = 0; x < R; ++x) if (!valid || k * R + x < first_row) ra[x] = __float_as_uint(-1e30f);
           }
-          float e_new[R], t_new[R];
+          uint64_t e_new[R / 2];
           const int c0 = (hl * W + k * R) / 2;               // pair index of this head's first column
 #pragma unroll
-          for (int x = 0; x < R; x += 2) {
-            const float4 c = coef[c0 + x / 2];                // (ref, ratio) of columns x and x + 1
-            t_new[x] = fmaf(__uint_as_float(ra[x]), p.sc2, -c.x);
-            t_new[x + 1] = fmaf(__uint_as_float(ra[x + 1]), p.sc2, -c.z);
+          for (int x = 0; x < R / 2; ++x) {
+            const float4 c = coef[c0 + x];                    // (-ref, -ref', ratio, ratio') of columns 2x and 2x + 1
+            float t0, t1;
+            f32x2_split(fma_f32x2(sm100::pack_f32x2(ra[2 * x], ra[2 * x + 1]), sc2x2, f32x2(c.x, c.y)), t0, t1);
+            e_new[x] = f32x2(fast_exp2(t0), fast_exp2(t1));
+            if (MODE == 1) { t_prev[2 * x] = t0; t_prev[2 * x + 1] = t1; }
           }
-#pragma unroll
-          for (int x = 0; x < R; ++x) e_new[x] = fast_exp2(t_new[x]);
           if (hl + 1 < heads) load(ra, hl + 1);              // the accumulators of this head are consumed
           if (MODE == 0) {
             if (hl > 0) consume(c0 - W / 2);
 #pragma unroll
-            for (int x = 0; x < R; ++x) e_prev[x] = valid ? e_new[x] : 0.f;
+            for (int x = 0; x < R / 2; ++x) e_prev[x] = e_new[x];
           } else {
             // the per-head entropies need the exponents as well: this mode (not the paper's default) takes
             // its sums at once rather than keep a second set of eight values for one head
 #pragma unroll
-            for (int x = 0; x < R; ++x) {
-              e_prev[x] = valid ? e_new[x] : 0.f;
-              t_prev[x] = t_new[x];
-            }
+            for (int x = 0; x < R / 2; ++x) e_prev[x] = e_new[x];
             consume(c0);
           }
         }
       }
       if (MODE == 0) consume(((heads - 1) * W + k * R) / 2);
+      float score;
+      {
+        float s0, s1;
+        f32x2_split(score2, s0, s1);
+        score = s0 + s1;
+      }
       // every column of the unit has been read: hand the accumulators back
       tc_fence_before_sync();
       __syncwarp();
@@ -371,10 +383,12 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 #pragma unroll
         for (int tt = 0; tt < 2; ++tt)
 #pragma unroll
-          for (int x = 0; x < R; ++x) {
-            const float a = abar[tt][x];
-            if (a > 0.f) acc = fmaf(a, __logf(a), acc);
-            abar[tt][x] = 0.f;
+          for (int x = 0; x < R / 2; ++x) {
+            float a0, a1;
+            f32x2_split(abar[tt][x], a0, a1);
+            if (a0 > 0.f) acc = fmaf(a0, __logf(a0), acc);
+            if (a1 > 0.f) acc = fmaf(a1, __logf(a1), acc);
+            abar[tt][x] = f32x2(0.f, 0.f);
           }
       }
       plogp = 0.f;
@@ -383,9 +397,11 @@ window_sweep_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         // one slot per 128-key tile and warp: an item's sum goes to its first tile, a zero to its second
         p.ent_partial[(size_t)(2 * blk + cur.t0) * kSwEpilogueWarps + ewarp] = acc;
         if (cur.nt > 1) p.ent_partial[(size_t)(2 * blk + 1) * kSwEpilogueWarps + ewarp] = 0.f;
-        __threadfence();
       }
     }
+    // once, after the last item (a fence after every item cost a twentieth of the sweep): the partials must be
+    // visible to the block that adds them up
+    if (p.ent_partial && lane == 0) __threadfence();
   }
 
   // ------------------------------------------------------------------ common exit

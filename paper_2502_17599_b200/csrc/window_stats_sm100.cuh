@@ -34,7 +34,7 @@
 namespace meda {
 
 constexpr int kWsStages = 6;
-constexpr int kWsEpilogueWarps = 8;                       // two groups of four: group t reduces row tile t
+constexpr int kWsEpilogueWarps = 16;                      // two groups of eight: group t reduces row tile t
 constexpr int kWsThreads = 32 * (2 + kWsEpilogueWarps);   // warp 0 TMA, warp 1 UMMA issue
 constexpr uint32_t kWsStageBytes = 2 * kUsHalfTile;       // 128 keys x 128 dims, bf16, two 64-column halves
 constexpr uint32_t kWsTmemCols = 512;
@@ -47,7 +47,7 @@ struct WinStatsParams {
   const __nv_bfloat16* q;        // [Hq * w][128]: window rows, head-major
   const uint8_t* modality;       // padded to a multiple of 128 with the value 2 (= no key)
   const uint32_t* tile_class;    // per 128-key tile: one byte per 32-key chunk: 0 all text, 1 all visual, 2 mixed / padding
-  float* partial;                // [Hq * w][chunks_pad][4]: a row's partials are contiguous (chunks_pad = chunks rounded up to 8)
+  float* partial;                // [chunks][Hq * w][4]: run-major, a warp's 32 rows of one run are contiguous
   float* row_stats;              // [Hq][w][4]  (written by the merging warps)
   float2* coef_vis;              // [Hq * w]    per-column constants of the second sweep, or null
   float2* coef_text;             // [Hq * w]
@@ -64,7 +64,8 @@ struct WinStatsSmem {
   static constexpr uint32_t bar_off = b_off + kWsStages * kWsStageBytes;
   static constexpr uint32_t n_bars = 2 * kWsStages + 2 * kWsSlots + 2;
   static constexpr uint32_t misc_off = bar_off + n_bars * 8;
-  static constexpr uint32_t total = misc_off + 16;
+  static constexpr uint32_t pair_off = misc_off + 16;                  // row states handed from a warp to its partner
+  static constexpr uint32_t total = pair_off + 8 * 32 * 16 + 8 * 4;
   static constexpr uint32_t alloc = total + 1024;         // slack for the manual 1024-byte alignment
 };
 
@@ -165,69 +166,101 @@ struct WinStatsRow {
   }
 };
 
+// (max, sum of exp2) of two disjoint key sets of a row, in base-2 logit units.
+__device__ __forceinline__ void merge_mz2(float& m, float& z, float m2, float z2) {
+  const float mn = fmaxf(m, m2);
+  if (mn == -INFINITY) { m = mn; z = 0.f; return; }
+  z = z * fast_exp2(m - mn) + z2 * fast_exp2(m2 - mn);
+  m = mn;
+}
+
 // Any chunk: per key modality (2 = no key) and visibility.  Only the few chunks where text and visual tokens
 // meet, the prompt's last keys (causal boundary) and the padding take this path; it is kept out of line, its
 // 32 logits passed through local memory, so that the code of the common path stays compact.  No tensor-memory
 // load may be in flight in the calling thread (a register that is saved around the call must hold its value).
+// Straight-line code: the maxima of the chunk's visible visual and text keys first, then one exponential per
+// key against its modality's maximum (taken key after key with a branch each, a single such chunk at the head of
+// the prompt held its block back by a fifth of the sweep).
 __device__ __noinline__ WinStatsRow win_stats_mixed_chunk(WinStatsRow s, const float* logits, float sc2, const uint8_t* mod32,
                                                           int j0, int last_visible) {
   // the chunk's 32 modality bytes in two loads (the map is padded and a chunk starts on a multiple of 32)
   const uint4 ma = __ldg(reinterpret_cast<const uint4*>(mod32)), mb = __ldg(reinterpret_cast<const uint4*>(mod32) + 1);
   const uint32_t mw[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+  uint32_t vis = 0u, text = 0u;               // bit x: key j0 + x is a visible visual / text key
 #pragma unroll
-  for (int w8 = 0; w8 < 8; ++w8) {
-#pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int x = 4 * w8 + b;
-      const int md = (int)((mw[w8] >> (8 * b)) & 0xffu);
-      if (md < 2 && j0 + x <= last_visible) {
-        if (md == MEDA_VISUAL) WinStatsRow::absorb(s.mv, s.zv, logits[x] * sc2);
-        else WinStatsRow::absorb(s.mt, s.zt, logits[x] * sc2);
-      }
-    }
+  for (int x = 0; x < 32; ++x) {
+    const uint32_t md = (mw[x / 4] >> (8 * (x % 4))) & 0xffu;
+    const bool seen = j0 + x <= last_visible;
+    vis |= (uint32_t)(seen && md == MEDA_VISUAL) << x;
+    text |= (uint32_t)(seen && md == MEDA_TEXT) << x;
   }
+  float mv = s.mv, mt = s.mt;
+#pragma unroll 4
+  for (int x = 0; x < 32; ++x) {
+    const float t = logits[x] * sc2;
+    mv = fmaxf(mv, (vis >> x) & 1u ? t : -INFINITY);
+    mt = fmaxf(mt, (text >> x) & 1u ? t : -INFINITY);
+  }
+  float zv = 0.f, zt = 0.f;
+#pragma unroll 4
+  for (int x = 0; x < 32; ++x) {
+    const float t = logits[x] * sc2;
+    const bool v = (vis >> x) & 1u, tx = (text >> x) & 1u;
+    const float e = (v || tx) ? fast_exp2(t - (v ? mv : mt)) : 0.f;
+    zv += v ? e : 0.f;
+    zt += tx ? e : 0.f;
+  }
+  // a modality without a key so far keeps (-inf, 0): its old sum is 0 and is not rescaled
+  s.zv = (s.zv > 0.f ? s.zv * fast_exp2(s.mv - mv) : 0.f) + zv;
+  s.zt = (s.zt > 0.f ? s.zt * fast_exp2(s.mt - mt) : 0.f) + zt;
+  s.mv = mv;
+  s.mt = mt;
   return s;
 }
 
-// Merges the partial normalisers of one query row over the key runs, in run order, and writes the row's
-// final normalisers and the two pairs of constants the second sweep uses for the row's column:
+#ifndef WS_MERGE_BATCH
+#define WS_MERGE_BATCH 6
+#endif
+// Partial normalisers of one query row over the key runs [c0, c1), merged in run order: a few runs at a time, their
+// maxima first and then the sums against that maximum, so that the exponentials of a batch do not wait for each
+// other.  `part` points at the row's entry of run 0; consecutive runs are `stride` entries apart (the layout is
+// run-major: the 32 rows of a warp read 512 contiguous bytes per run).  Natural-log units.
+// Returns (m, z, m_vis, z_vis).
+__device__ __forceinline__ float4 win_stats_merge_runs(const float4* part, size_t stride, int c0, int c1) {
+  float m = -INFINITY, mv = -INFINITY, z = 0.f, zv = 0.f;
+  constexpr int kBatch = WS_MERGE_BATCH;
+#pragma unroll 1
+  for (int cb = c0; cb < c1; cb += kBatch) {
+    float4 x[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u)
+      x[u] = (cb + u < c1) ? __ldcg(part + (size_t)(cb + u) * stride) : make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
+    float mb = -INFINITY, mvb = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      mb = fmaxf(mb, x[u].x);
+      mvb = fmaxf(mvb, x[u].z);
+    }
+    float zb = 0.f, zvb = 0.f;
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      // a run without a visible (visual) key has the sum 0 and the maximum -inf
+      zb += x[u].y > 0.f ? x[u].y * __expf(x[u].x - mb) : 0.f;
+      zvb += x[u].w > 0.f ? x[u].w * __expf(x[u].z - mvb) : 0.f;
+    }
+    merge_mz(m, z, mb, zb);
+    merge_mz(mv, zv, mvb, zvb);
+  }
+  return make_float4(m, z, mv, zv);
+}
+
+// Writes a row's final normalisers and the two pairs of constants the second sweep uses for the row's column:
 //   vis  = (m_vis * log2e + log2(z_vis * Hq),  Hq * z_vis * exp(m_vis - m_all) / z_all)   for visual keys
 //   text = (m_all * log2e,                     1 / z_all)                                 for text keys
 // (a row that sees no visual key gets (+huge, 0): its exponentials are 0).
-__device__ __forceinline__ void win_stats_finish_row(const WinStatsParams& p, int h, int i) {
+__device__ __forceinline__ void win_stats_write_row(const WinStatsParams& p, int h, int i, float m, float z, float mv,
+                                                    float zv) {
   const size_t row = (size_t)h * p.w + i;
-  const int chunks_pad = (p.chunks + 7) / 8 * 8;
-  const float4* part = reinterpret_cast<const float4*>(p.partial) + row * chunks_pad;
-  // The row's partials lie in a few consecutive 128-byte lines, written by other blocks (this block has not read
-  // them before, and the first-level cache holds nothing from earlier launches).  One load per line goes out first,
-  // so that all lines travel at once; the rest of each line then comes at cache speed.  Each line's eight partials
-  // are merged as a fixed tree and the lines in order: the dependent chain is a few merges long instead of one per
-  // key run, and the result depends on nothing but the data.
-  constexpr int kLines = (kWsMaxChunks + 7) / 8;
-  const float4 nothing = make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
-  float4 head[kLines];
-#pragma unroll
-  for (int b = 0; b < kLines; ++b) head[b] = (8 * b < p.chunks) ? part[8 * b] : nothing;
-  float m = -INFINITY, z = 0.f, mv = -INFINITY, zv = 0.f;
-#pragma unroll
-  for (int b = 0; b < kLines; ++b) {
-    if (8 * b < p.chunks) {
-      float4 x[8];
-      x[0] = head[b];
-#pragma unroll
-      for (int u = 1; u < 8; ++u) x[u] = (8 * b + u < p.chunks) ? part[8 * b + u] : nothing;
-#pragma unroll
-      for (int step = 1; step < 8; step <<= 1) {
-#pragma unroll
-        for (int u = 0; u < 8; u += 2 * step) {
-          merge_mz(x[u].x, x[u].y, x[u + step].x, x[u + step].y);
-          merge_mz(x[u].z, x[u].w, x[u + step].z, x[u + step].w);
-        }
-      }
-      merge_mz(m, z, x[0].x, x[0].y);
-      merge_mz(mv, zv, x[0].z, x[0].w);
-    }
-  }
   reinterpret_cast<float4*>(p.row_stats)[row] = make_float4(m, z, mv, zv);
   if (p.coef_vis) {
     float2 a = make_float2(1e30f, 0.f);
@@ -260,7 +293,7 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kWsStages; ++s) { mbar_init(b_full + s, 1); mbar_init(b_empty + s, 1); }
-    for (uint32_t s = 0; s < kWsSlots; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, 4); }
+    for (uint32_t s = 0; s < kWsSlots; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, kWsEpilogueWarps / 2); }
     mbar_init(a_ready, kWsEpilogueWarps);
     mbar_init(a_free, 1);
     *abort_flag = 0;
@@ -332,9 +365,14 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
     }
   } else {
     // ------------------------------------------------------------------ epilogue (and loader of the query rows)
+    // Warp (t, quarter, half): row tile t, tensor-memory lanes of `quarter`, chunks 2 half and 2 half + 1 of every
+    // unit.  Four epilogue warps per scheduler: while one waits for its accumulators the others keep the
+    // special-function unit busy.
     const int ewarp = warp - 2;
-    const int t = ewarp / 4;                    // row tile = epilogue group
+    const int t = (ewarp / 4) & 1;              // row tile = epilogue group
+    const int half = ewarp / 8;                 // which two of a unit's four 32-key chunks
     const int quarter = warp % 4;               // tensor-memory lanes this warp may touch: 32 * (warp % 4) ..
+    const int set = t * 4 + ewarp % 4;          // the 32 rows this warp shares with its partner (the other half)
     const int row_in_block = t * 128 + quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     WinStatsRow row;
@@ -345,23 +383,20 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
       const int r = it.rb * 256 + row_in_block;     // query row inside the KV group
       const bool mine = t < it.m_tiles;
       const bool valid = mine && r < p.cols;
-      // ---- this thread's query row -> tensor memory, once the previous item's UMMAs are done with it
+      // ---- half of this thread's query row -> tensor memory, once the previous item's UMMAs are done with it
       ok = mbar_wait(a_free, (item & 1u) ^ 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after_sync();
       if (mine) {
         const uint4* src = reinterpret_cast<const uint4*>(p.q + ((size_t)it.g * p.cols + min(r, p.cols - 1)) * kFastDim);
+        uint32_t a[32];
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t a[32];
-#pragma unroll
-          for (int x = 0; x < 8; ++x) {
-            const uint4 v = valid ? __ldg(src + half * 8 + x) : make_uint4(0u, 0u, 0u, 0u);
-            a[4 * x + 0] = v.x; a[4 * x + 1] = v.y; a[4 * x + 2] = v.z; a[4 * x + 3] = v.w;
-          }
-          tmem_st_32x32(lane_addr + (uint32_t)t * 64u + (uint32_t)half * 32u, a);
+        for (int x = 0; x < 8; ++x) {
+          const uint4 v = valid ? __ldg(src + half * 8 + x) : make_uint4(0u, 0u, 0u, 0u);
+          a[4 * x + 0] = v.x; a[4 * x + 1] = v.y; a[4 * x + 2] = v.z; a[4 * x + 3] = v.w;
         }
+        tmem_st_32x32(lane_addr + (uint32_t)t * 64u + (uint32_t)half * 32u, a);
         tmem_st_wait();
       }
       tc_fence_before_sync();
@@ -384,59 +419,30 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t taddr = lane_addr + kWsAccBase + slot * 128u;
-          const int c0 = it.b_row + tile * 128;
-          // Two register buffers: the load of chunk c + 1 is in flight while chunk c is reduced, except around
-          // the out-of-line path, which runs with nothing in flight.
-          uint32_t ra[32], rb[32];
-          tmem_ld_32x32_issue(taddr, ra);
+          const uint32_t taddr = lane_addr + kWsAccBase + slot * 128u + (uint32_t)half * 64u;
+          const int c0 = it.b_row + tile * 128 + half * 64;
+          uint32_t ra[32];
 #pragma unroll 1
-          for (int c = 0; c < 4; c += 2) {
-            {
-              tmem_ld_wait();
-              tmem_ld_pin(ra);
-              const uint32_t cl = (cls_now >> (8 * c)) & 0xffu;
-              const int j0 = c0 + 32 * c;
-              // uniform over the warp: the branches below hold warp-wide (.sync.aligned) tensor-memory loads
-              const bool fast = __all_sync(0xffffffffu, !valid || (cl < 2u && j0 + 31 <= last_visible));
-              if (fast) {
-                tmem_ld_32x32_issue(taddr + 32u * (c + 1), rb);
-                if (valid) row.uniform_chunk(ra, p.sc2, cl == 1u);
-              } else {
-                if (valid) {
-                  float tmp[32];
-#pragma unroll
-                  for (int x = 0; x < 32; ++x) tmp[x] = __uint_as_float(ra[x]);
-                  row = win_stats_mixed_chunk(row, tmp, p.sc2, p.modality + j0, j0, last_visible);
-                }
-                tmem_ld_32x32_issue(taddr + 32u * (c + 1), rb);
-              }
+          for (int c = 0; c < 2; ++c) {
+            tmem_ld_32x32_issue(taddr + 32u * c, ra);
+            tmem_ld_wait();
+            tmem_ld_pin(ra);
+            if (c == 1) {
+              // this warp's share of the unit is in registers: hand the slot back before the last chunk is reduced
+              tc_fence_before_sync();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(s_empty + slot);
             }
-            {
-              tmem_ld_wait();
-              tmem_ld_pin(rb);
-              const uint32_t cl = (cls_now >> (8 * (c + 1))) & 0xffu;
-              const int j0 = c0 + 32 * (c + 1);
-              // uniform over the warp: the branches below hold warp-wide (.sync.aligned) tensor-memory loads
-              const bool fast = __all_sync(0xffffffffu, !valid || (cl < 2u && j0 + 31 <= last_visible));
-              if (c == 2) {
-                // the whole unit is in registers: hand the slot back before the last chunk is reduced
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(s_empty + slot);
-              }
-              if (fast) {
-                if (c == 0) tmem_ld_32x32_issue(taddr + 64u, ra);
-                if (valid) row.uniform_chunk(rb, p.sc2, cl == 1u);
-              } else {
-                if (valid) {
-                  float tmp[32];
+            const uint32_t cl = (cls_now >> (8 * (2 * half + c))) & 0xffu;
+            const int j0 = c0 + 32 * c;
+            const bool fast = __all_sync(0xffffffffu, !valid || (cl < 2u && j0 + 31 <= last_visible));
+            if (fast) {
+              if (valid) row.uniform_chunk(ra, p.sc2, cl == 1u);
+            } else if (valid) {
+              float tmp[32];
 #pragma unroll
-                  for (int x = 0; x < 32; ++x) tmp[x] = __uint_as_float(rb[x]);
-                  row = win_stats_mixed_chunk(row, tmp, p.sc2, p.modality + j0, j0, last_visible);
-                }
-                if (c == 0) tmem_ld_32x32_issue(taddr + 64u, ra);
-              }
+              for (int x = 0; x < 32; ++x) tmp[x] = __uint_as_float(ra[x]);
+              row = win_stats_mixed_chunk(row, tmp, p.sc2, p.modality + j0, j0, last_visible);
             }
           }
         }
@@ -444,25 +450,55 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
       if (!ok) break;
       unit_base += (uint32_t)(it.n_tiles * it.m_tiles);
 
-      // ---- partial normalisers of the item; the warp that completes its 32 rows merges them
-      if (mine) {
+      // ---- the two halves of a row meet in the half-0 warp (through shared memory, a 64-thread barrier per set)
+      float4* pair_state = reinterpret_cast<float4*>(smem + SH::pair_off) + set * 32 + lane;
+      volatile int* pair_flag = reinterpret_cast<volatile int*>(smem + SH::pair_off + 8 * 32 * 16) + set;
+      if (half == 1) *pair_state = make_float4(row.mv, row.zv, row.mt, row.zt);
+      asm volatile("bar.sync %0, 64;" ::"r"(1 + set) : "memory");
+      if (half == 0) {
+        const float4 o = *pair_state;
+        merge_mz2(row.mv, row.zv, o.x, o.y);
+        merge_mz2(row.mt, row.zt, o.z, o.w);
+      }
+
+      // ---- partial normalisers of the item; the pair of warps that completes its 32 rows merges them
+      const size_t rows_total = (size_t)p.hq * p.w;
+      const int h = it.g * p.group + min(r, p.cols - 1) / p.w;
+      float4* my_part = reinterpret_cast<float4*>(p.partial) + (size_t)h * p.w + i_win;     // run 0 of this row
+      unsigned int* counter = p.counters + ((size_t)(it.g * p.row_blocks + it.rb) * 8 + set);
+      bool last = false;
+      if (mine && half == 0) {
         if (valid) {
-          const int h = it.g * p.group + r / p.w;
           const float m_all = fmaxf(row.mv, row.mt);
           float z_all = 0.f;
           if (m_all > -INFINITY) z_all = row.zv * fast_exp2(row.mv - m_all) + row.zt * fast_exp2(row.mt - m_all);
-          reinterpret_cast<float4*>(p.partial)[((size_t)h * p.w + i_win) * ((p.chunks + 7) / 8 * 8) + it.kc] =
-              make_float4(m_all * kLn2, z_all, row.mv * kLn2, row.zv);
+          my_part[(size_t)it.kc * rows_total] = make_float4(m_all * kLn2, z_all, row.mv * kLn2, row.zv);
         }
         __threadfence();
         __syncwarp();
         unsigned int ticket = 0;
-        unsigned int* counter = p.counters + ((size_t)(it.g * p.row_blocks + it.rb) * kWsEpilogueWarps + ewarp);
         if (lane == 0) ticket = atomicAdd(counter, 1u);
         ticket = __shfl_sync(0xffffffffu, ticket, 0);
-        if (ticket == (unsigned int)p.chunks - 1u) {       // every key run of these rows has been written
-          __threadfence();
-          if (valid) win_stats_finish_row(p, it.g * p.group + r / p.w, i_win);
+        last = ticket == (unsigned int)p.chunks - 1u;      // every key run of these rows has been written
+        if (lane == 0) *pair_flag = last ? 1 : 0;
+      }
+      asm volatile("bar.sync %0, 64;" ::"r"(1 + set) : "memory");
+      last = *pair_flag != 0;                              // uniform over the pair of warps
+      if (last) {
+        // each warp of the pair merges half of the key runs, the half-0 warp joins the halves and writes the row
+        __threadfence();
+        const int c_mid = (p.chunks + 1) / 2;
+        float4 mine4 = make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
+        if (valid) mine4 = win_stats_merge_runs(my_part, rows_total, half ? c_mid : 0, half ? p.chunks : c_mid);
+        if (half == 1) *pair_state = mine4;
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + set) : "memory");
+        if (half == 0) {
+          if (valid) {
+            const float4 o = *pair_state;
+            merge_mz(mine4.x, mine4.y, o.x, o.y);
+            merge_mz(mine4.z, mine4.w, o.z, o.w);
+            win_stats_write_row(p, h, i_win, mine4.x, mine4.y, mine4.z, mine4.w);
+          }
           if (lane == 0) *counter = 0u;                    // ready for the next launch
         }
       }

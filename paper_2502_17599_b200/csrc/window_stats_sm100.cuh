@@ -175,51 +175,58 @@ __device__ __forceinline__ void merge_mz2(float& m, float& z, float m2, float z2
 }
 
 // Any chunk: per key modality (2 = no key) and visibility.  Only the few chunks where text and visual tokens
-// meet, the prompt's last keys (causal boundary) and the padding take this path; it is kept out of line, its
-// 32 logits passed through local memory, so that the code of the common path stays compact.  No tensor-memory
-// load may be in flight in the calling thread (a register that is saved around the call must hold its value).
-// Straight-line code: the maxima of the chunk's visible visual and text keys first, then one exponential per
-// key against its modality's maximum (taken key after key with a branch each, a single such chunk at the head of
-// the prompt held its block back by a fifth of the sweep).
-__device__ __noinline__ WinStatsRow win_stats_mixed_chunk(WinStatsRow s, const float* logits, float sc2, const uint8_t* mod32,
-                                                          int j0, int last_visible) {
-  // the chunk's 32 modality bytes in two loads (the map is padded and a chunk starts on a multiple of 32)
-  const uint4 ma = __ldg(reinterpret_cast<const uint4*>(mod32)), mb = __ldg(reinterpret_cast<const uint4*>(mod32) + 1);
-  const uint32_t mw[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
-  uint32_t vis = 0u, text = 0u;               // bit x: key j0 + x is a visible visual / text key
+// meet, the prompt's last keys (causal boundary) and the padding take this path.  It reads the chunk's
+// accumulators itself, eight columns at a time and twice (the maxima of the chunk's visible visual and text keys
+// first, then one exponential per key against its modality's maximum), in rolled loops: little code, few
+// registers, nothing in local memory.  (Taken key after key with a branch each, or through an array in local
+// memory, a single such chunk at the head of the prompt held its block back by a sixth of the sweep.)
+// Warp-wide: every lane must call it (tensor-memory loads are .sync.aligned); `valid` lanes update their row.
+// `vis_keys` / `text_keys`: bit x set when key j0 + x is a visual / text key (the same for every row); the row's
+// own causal limit masks them.
+__device__ __forceinline__ void win_stats_mixed_chunk(WinStatsRow& s, bool valid, uint32_t taddr, float sc2, uint32_t vis_keys,
+                                                      uint32_t text_keys, int j0, int last_visible) {
+  const int n_seen = min(max(last_visible - j0 + 1, 0), 32);
+  const uint32_t seen = n_seen >= 32 ? 0xffffffffu : ((1u << n_seen) - 1u);
+  const uint32_t vis = valid ? vis_keys & seen : 0u, text = valid ? text_keys & seen : 0u;
+  // maxima on the raw accumulators (the scale is positive), scaled once
+  float rv = -INFINITY, rt = -INFINITY;
+#pragma unroll 1
+  for (int x0 = 0; x0 < 32; x0 += 8) {
+    uint32_t r[8];
+    sm100::tmem_ld_32x8_issue(taddr + (uint32_t)x0, r);
+    sm100::tmem_ld_wait();
+    sm100::tmem_ld_pin_n<8>(r);
 #pragma unroll
-  for (int x = 0; x < 32; ++x) {
-    const uint32_t md = (mw[x / 4] >> (8 * (x % 4))) & 0xffu;
-    const bool seen = j0 + x <= last_visible;
-    vis |= (uint32_t)(seen && md == MEDA_VISUAL) << x;
-    text |= (uint32_t)(seen && md == MEDA_TEXT) << x;
+    for (int x = 0; x < 8; ++x) {
+      rv = fmaxf(rv, (vis >> (x0 + x)) & 1u ? __uint_as_float(r[x]) : -INFINITY);
+      rt = fmaxf(rt, (text >> (x0 + x)) & 1u ? __uint_as_float(r[x]) : -INFINITY);
+    }
   }
-  float mv = s.mv, mt = s.mt;
-#pragma unroll 4
-  for (int x = 0; x < 32; ++x) {
-    const float t = logits[x] * sc2;
-    mv = fmaxf(mv, (vis >> x) & 1u ? t : -INFINITY);
-    mt = fmaxf(mt, (text >> x) & 1u ? t : -INFINITY);
-  }
+  const float mv = fmaxf(s.mv, rv * sc2), mt = fmaxf(s.mt, rt * sc2);
   float zv = 0.f, zt = 0.f;
-#pragma unroll 4
-  for (int x = 0; x < 32; ++x) {
-    const float t = logits[x] * sc2;
-    const bool v = (vis >> x) & 1u, tx = (text >> x) & 1u;
-    const float e = (v || tx) ? fast_exp2(t - (v ? mv : mt)) : 0.f;
-    zv += v ? e : 0.f;
-    zt += tx ? e : 0.f;
+#pragma unroll 1
+  for (int x0 = 0; x0 < 32; x0 += 8) {
+    uint32_t r[8];
+    sm100::tmem_ld_32x8_issue(taddr + (uint32_t)x0, r);
+    sm100::tmem_ld_wait();
+    sm100::tmem_ld_pin_n<8>(r);
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+      const bool v = (vis >> (x0 + x)) & 1u, tx = (text >> (x0 + x)) & 1u;
+      const float e = (v || tx) ? fast_exp2(fmaf(__uint_as_float(r[x]), sc2, v ? -mv : -mt)) : 0.f;
+      zv += v ? e : 0.f;
+      zt += tx ? e : 0.f;
+    }
   }
   // a modality without a key so far keeps (-inf, 0): its old sum is 0 and is not rescaled
   s.zv = (s.zv > 0.f ? s.zv * fast_exp2(s.mv - mv) : 0.f) + zv;
   s.zt = (s.zt > 0.f ? s.zt * fast_exp2(s.mt - mt) : 0.f) + zt;
   s.mv = mv;
   s.mt = mt;
-  return s;
 }
 
 #ifndef WS_MERGE_BATCH
-#define WS_MERGE_BATCH 6
+#define WS_MERGE_BATCH 10
 #endif
 // Partial normalisers of one query row over the key runs [c0, c1), merged in run order: a few runs at a time, their
 // maxima first and then the sums against that maximum, so that the exponentials of a batch do not wait for each
@@ -424,26 +431,27 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
           uint32_t ra[32];
 #pragma unroll 1
           for (int c = 0; c < 2; ++c) {
-            tmem_ld_32x32_issue(taddr + 32u * c, ra);
-            tmem_ld_wait();
-            tmem_ld_pin(ra);
+            const uint32_t cl = (cls_now >> (8 * (2 * half + c))) & 0xffu;
+            const int j0 = c0 + 32 * c;
+            // uniform over the warp: the branches below hold warp-wide (.sync.aligned) tensor-memory loads
+            const bool fast = __all_sync(0xffffffffu, !valid || (cl < 2u && j0 + 31 <= last_visible));
+            if (fast) {
+              tmem_ld_32x32_issue(taddr + 32u * c, ra);
+              tmem_ld_wait();
+              tmem_ld_pin(ra);
+            } else {
+              const int md = p.modality[j0 + lane];          // the map is padded: 2 = no key
+              const uint32_t vis_keys = __ballot_sync(0xffffffffu, md == MEDA_VISUAL);
+              const uint32_t text_keys = __ballot_sync(0xffffffffu, md == MEDA_TEXT);
+              win_stats_mixed_chunk(row, valid, taddr + 32u * c, p.sc2, vis_keys, text_keys, j0, last_visible);
+            }
             if (c == 1) {
-              // this warp's share of the unit is in registers: hand the slot back before the last chunk is reduced
+              // this warp's share of the unit has been read: hand the slot back before the last chunk is reduced
               tc_fence_before_sync();
               __syncwarp();
               if (lane == 0) mbar_arrive(s_empty + slot);
             }
-            const uint32_t cl = (cls_now >> (8 * (2 * half + c))) & 0xffu;
-            const int j0 = c0 + 32 * c;
-            const bool fast = __all_sync(0xffffffffu, !valid || (cl < 2u && j0 + 31 <= last_visible));
-            if (fast) {
-              if (valid) row.uniform_chunk(ra, p.sc2, cl == 1u);
-            } else if (valid) {
-              float tmp[32];
-#pragma unroll
-              for (int x = 0; x < 32; ++x) tmp[x] = __uint_as_float(ra[x]);
-              row = win_stats_mixed_chunk(row, tmp, p.sc2, p.modality + j0, j0, last_visible);
-            }
+            if (fast && valid) row.uniform_chunk(ra, p.sc2, cl == 1u);
           }
         }
       }

@@ -4,25 +4,29 @@
 // One persistent block per SM.  An item is (KV group, block of up to 256 query rows, run of 128-key tiles).
 //
 //  * The query rows are the A operand of the UMMAs and live in TENSOR MEMORY for the whole item (each
-//    epilogue thread loads its own row once and stores it with tcgen05.st): the tensor pipe then reads only
+//    epilogue thread loads half of its row once and stores it with tcgen05.st): the tensor pipe then reads only
 //    the streamed key tile from shared memory.  With both operands in shared memory the operand reads of a
 //    128 x 128 x 16 instruction take as long as its arithmetic, and the kernel with an empty epilogue already
 //    ran well above the time the keys need to arrive.
 //  * Key tiles (128 keys) arrive by TMA through a six-stage ring.
 //  * Accumulators are handed over per UNIT = (128-row tile, key tile), 128 columns each, through three
-//    rotating slots of tensor memory.  Epilogue group t (four warps, one per lane quarter) owns row tile t
-//    and therefore every other unit; with three slots the tensor pipe always has a free slot to fill while
-//    both groups are reducing, so neither waits for the other nor for the UMMAs of its next unit.
-//  * Every epilogue thread owns one query row and keeps online (max, sum of exp2) over visual and over text
-//    keys.  Per 32-key chunk: the chunk maximum by three-input maxima, then one exponential per logit.
-//    Exponentials are the scarcest resource here (one per logit on 16 special-function lanes per SM), so a
-//    fixed share of every chunk is evaluated on the FMA pipes instead: round-to-nearest split of the
-//    exponent, degree-5 polynomial in packed pairs, exponent added as an integer (relative error 2.4e-7,
-//    the special-function unit's own is 1.7e-7).
-//  * The partial normalisers of an item go to global memory; the warp that completes a set of 32 rows over
-//    all key runs (counted with one atomic per warp and item) merges them in key-run order and writes the
-//    rows' final normalisers together with the per-column constants the second sweep reads.  Which warp
-//    does it depends on timing; what it computes does not.
+//    rotating slots of tensor memory.  Epilogue group t (eight warps: two per lane quarter, each taking two of
+//    the unit's four 32-key chunks) owns row tile t and therefore every other unit; with three slots the tensor
+//    pipe always has a free slot to fill while both groups are reducing.  Four epilogue warps per scheduler:
+//    while one waits for its accumulators the others keep the special-function unit busy (with two per
+//    scheduler a warp's chunk took 650 cycles against the 512 the unit needs for two warps' exponentials).
+//  * Every epilogue thread owns one query row for two chunks of every unit and keeps online (max, sum of exp2)
+//    over visual and over text keys.  Per 32-key chunk: the chunk maximum by three-input maxima, then one
+//    exponential per logit on the special-function unit.  A share of the exponentials can be moved to the FMA
+//    pipes (exp2_poly_pair: round-to-nearest split of the exponent, degree-5 polynomial in packed pairs,
+//    exponent added as an integer; relative error 2.4e-7, the special-function unit's own is 1.7e-7).  That paid
+//    with two epilogue warps per scheduler (a quarter of the exponentials: 5 %); with four the sweep is short of
+//    issue slots rather than of exponentials and the share is zero (a quarter: +4 % time, half: +12 %).
+//  * The two warps that share a row add their states through shared memory at the end of an item.  The
+//    partial normalisers of an item go to global memory, run-major; the pair of warps that completes a set of 32
+//    rows over all key runs (counted with one atomic per pair and item) merges them, each warp half of the
+//    runs, in run order, and writes the rows' final normalisers together with the per-column constants the
+//    second sweep reads.  Which pair does it depends on timing; what it computes does not.
 //
 // Logits are kept in base-2 units: t = (q.k) * scale * log2(e).
 #pragma once
@@ -41,7 +45,7 @@ constexpr uint32_t kWsTmemCols = 512;
 constexpr uint32_t kWsAccBase = 128;                      // columns [0, 128): the query rows, 64 per row tile
 constexpr uint32_t kWsSlots = 3;                          // accumulator slots of 128 columns
 constexpr int kWsMaxChunks = 64;                          // key runs per (KV group, row block): at most this many partials per row
-constexpr int kWsPolyOf8 = 2;                             // exponentials per 8 that take the FMA pipes
+constexpr int kWsPolyOf8 = 0;                             // exponentials per 8 that take the FMA pipes (none: see below)
 
 struct WinStatsParams {
   const __nv_bfloat16* q;        // [Hq * w][128]: window rows, head-major
@@ -127,14 +131,17 @@ struct WinStatsRow {
   }
   // 32 consecutive keys of one modality, all visible: the chunk maximum first, then one exponential per key.
   __device__ __forceinline__ void uniform_chunk(const uint32_t (&r)[32], float sc2, bool visual) {
-    float t[12];
+    // four independent chains of three-input maxima
+    float u0 = __uint_as_float(r[0]), u1 = __uint_as_float(r[1]), u2 = __uint_as_float(r[2]), u3 = __uint_as_float(r[3]);
 #pragma unroll
-    for (int x = 0; x < 10; ++x)
-      t[x] = sm100::fmax3(__uint_as_float(r[3 * x]), __uint_as_float(r[3 * x + 1]), __uint_as_float(r[3 * x + 2]));
-    t[10] = __uint_as_float(r[30]);
-    t[11] = __uint_as_float(r[31]);
-    const float u0 = sm100::fmax3(t[0], t[1], t[2]), u1 = sm100::fmax3(t[3], t[4], t[5]);
-    const float u2 = sm100::fmax3(t[6], t[7], t[8]), u3 = sm100::fmax3(t[9], t[10], t[11]);
+    for (int x = 4; x < 28; x += 8) {
+      u0 = sm100::fmax3(u0, __uint_as_float(r[x]), __uint_as_float(r[x + 1]));
+      u1 = sm100::fmax3(u1, __uint_as_float(r[x + 2]), __uint_as_float(r[x + 3]));
+      u2 = sm100::fmax3(u2, __uint_as_float(r[x + 4]), __uint_as_float(r[x + 5]));
+      u3 = sm100::fmax3(u3, __uint_as_float(r[x + 6]), __uint_as_float(r[x + 7]));
+    }
+    u0 = sm100::fmax3(u0, __uint_as_float(r[28]), __uint_as_float(r[29]));
+    u1 = sm100::fmax3(u1, __uint_as_float(r[30]), __uint_as_float(r[31]));
     const float cm = fmaxf(sm100::fmax3(u0, u1, u2), u3);
     float& m = visual ? mv : mt;
     float& z = visual ? zv : zt;
@@ -157,6 +164,9 @@ struct WinStatsRow {
         }
         if (pr & 1) a23 = add_f32x2(a23, e); else a01 = add_f32x2(a01, e);
       }
+      // the sums so far are complete here: keeps the compiler from issuing all 32 exponentials before the first
+      // addition, which needs more registers than a thread of this block can have
+      asm volatile("" : "+l"(a01), "+l"(a23));
     }
     float a0, a1, a2, a3;
     f32x2_split(a01, a0, a1);
@@ -226,7 +236,7 @@ __device__ __forceinline__ void win_stats_mixed_chunk(WinStatsRow& s, bool valid
 }
 
 #ifndef WS_MERGE_BATCH
-#define WS_MERGE_BATCH 10
+#define WS_MERGE_BATCH 8
 #endif
 // Partial normalisers of one query row over the key runs [c0, c1), merged in run order: a few runs at a time, their
 // maxima first and then the sums against that maximum, so that the exponentials of a batch do not wait for each
@@ -473,7 +483,6 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
       const size_t rows_total = (size_t)p.hq * p.w;
       const int h = it.g * p.group + min(r, p.cols - 1) / p.w;
       float4* my_part = reinterpret_cast<float4*>(p.partial) + (size_t)h * p.w + i_win;     // run 0 of this row
-      unsigned int* counter = p.counters + ((size_t)(it.g * p.row_blocks + it.rb) * 8 + set);
       bool last = false;
       if (mine && half == 0) {
         if (valid) {
@@ -485,7 +494,7 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
         __threadfence();
         __syncwarp();
         unsigned int ticket = 0;
-        if (lane == 0) ticket = atomicAdd(counter, 1u);
+        if (lane == 0) ticket = atomicAdd(p.counters + ((size_t)(it.g * p.row_blocks + it.rb) * 8 + set), 1u);
         ticket = __shfl_sync(0xffffffffu, ticket, 0);
         last = ticket == (unsigned int)p.chunks - 1u;      // every key run of these rows has been written
         if (lane == 0) *pair_flag = last ? 1 : 0;
@@ -507,7 +516,7 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
             merge_mz(mine4.z, mine4.w, o.z, o.w);
             win_stats_write_row(p, h, i_win, mine4.x, mine4.y, mine4.z, mine4.w);
           }
-          if (lane == 0) *counter = 0u;                    // ready for the next launch
+          if (lane == 0) p.counters[(size_t)(it.g * p.row_blocks + it.rb) * 8 + set] = 0u;     // ready for the next launch
         }
       }
     }

@@ -286,9 +286,10 @@ CSRC = "paper_2502_17599_b200/csrc/"
 KERNEL_TRAFFIC = {
     # class: (bytes per launch, source files, sha256[:16] of their concatenation)
     "nearest": (138.9e6, (CSRC + "nearest_sm100.cuh", CSRC + "sm100_primitives.cuh"), "802a52cd62a33938"),
-    "stats": (136.8e6, (CSRC + "window_stats_sm100.cuh", CSRC + "sm100_primitives.cuh"), "8796929e3a0b9995"),
-    "sweep": (137.3e6, (CSRC + "window_sweep_sm100.cuh", CSRC + "sm100_primitives.cuh"), "73e64b1d83362859"),
-    "reduce": (288.1e6, (CSRC + "group_reduce.cuh",), "71af809bda69dc5b"),
+    "stats": (136.8e6, (CSRC + "window_stats_sm100.cuh", CSRC + "attn_sm100.cuh", CSRC + "sm100_primitives.cuh"), "c8b650b1da4d04ef"),
+    "sweep": (136.8e6, (CSRC + "window_sweep_sm100.cuh", CSRC + "window_stats_sm100.cuh", CSRC + "attn_sm100.cuh",
+                        CSRC + "sm100_primitives.cuh"), "89fd96e6dce1480c"),
+    "reduce": (288.8e6, (CSRC + "group_reduce.cuh",), "9a2cd791f2d0ea71"),
 }
 NOMINAL_HBM_GBS = 8000.0     # the nominal figure the target is worded against; the measured copy peak is the denominator of `frac`
 

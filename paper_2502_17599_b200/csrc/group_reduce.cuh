@@ -26,7 +26,7 @@ constexpr int kSortBlockItems = kSortWarps * kSortWarpItems; // elements of one 
 constexpr int kSegChunk = 128;        // sorted rows walked by one warp
 constexpr int kSegWarps = 2;         // small blocks: more of them fit, also beside a resident tensor-core block
 
-// ---- stable radix pass: histogram, scan, scatter ----------------------------------------------
+// ---- stable radix pass: histogram, scatter ----------------------------------------------------
 // The keys are slots < S, so the pass over the digit at `shift` orders nothing when S <= 2^shift: its three
 // kernels return at once (the host enqueues the passes the prompt length may need; the layer's budget is only
 // known on the device) and the consumer picks the buffer the last executed pass wrote.
@@ -70,58 +70,14 @@ sort_hist_kernel(const int32_t* __restrict__ keys, const int32_t* __restrict__ b
   for (int b = threadIdx.x; b < kSortBins; b += blockDim.x) tg[(size_t)b * n_blocks + blk] = cnt[b];
 }
 
-// In-place exclusive prefix sum of each head's table in (bin, chunk) order.  One block per head;
-// `len` is a multiple of 4096 (the chunk count is padded to a multiple of 8), so every thread owns
-// a run of len / 1024 entries that is a whole number of 16-byte vectors.
-__global__ void __launch_bounds__(1024)
-sort_scan_kernel(int32_t* __restrict__ table, int len, const int32_t* __restrict__ budget_row, int cap, int shift) {
-  __shared__ int warp_sums[32];
-  if (!sort_pass_needed(min(budget_row[0], cap), shift)) return;
-  int4* t = reinterpret_cast<int4*>(table + (size_t)blockIdx.x * len);
-  const int per = len / 4096;                         // vectors per thread
-  const int begin = (int)threadIdx.x * per;
-  int sum = 0;
-  for (int e0 = 0; e0 < per; e0 += 8) {
-    int4 x[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) x[u] = (e0 + u < per) ? t[begin + e0 + u] : make_int4(0, 0, 0, 0);
-#pragma unroll
-    for (int u = 0; u < 8; ++u) sum += x[u].x + x[u].y + x[u].z + x[u].w;
-  }
-  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-  int incl = sum;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += y;
-  }
-  if (lane == 31) warp_sums[warp] = incl;
-  __syncthreads();
-  if (warp == 0) {
-    int w = warp_sums[lane], wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int y = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += y;
-    }
-    warp_sums[lane] = wi - w;
-  }
-  __syncthreads();
-  int run = warp_sums[warp] + incl - sum;
-  for (int e = 0; e < per; ++e) {
-    int4 x = t[begin + e], y;
-    y.x = run; run += x.x;
-    y.y = run; run += x.y;
-    y.z = run; run += x.z;
-    y.w = run; run += x.w;
-    t[begin + e] = y;
-  }
-}
-
-// Stable scatter of (key, row) pairs by the digit at `shift`, using the scanned table.  Inside a block
-// the eight warps own consecutive runs of 256 elements: each first counts its digits, the counts are
-// turned into per-warp start offsets (block base from the table + the earlier warps' counts), then every
-// warp ranks its elements in index order.
+// Stable scatter of (key, row) pairs by the digit at `shift`.  A block's first output position for a digit is
+// the number of keys with a smaller digit anywhere plus the number with this digit in earlier blocks: every
+// block takes both from the digit table itself (512 rows of one count per block, 128 KB per head, resident in L2:
+// a row's total and its prefix up to this block, then a block-wide exclusive scan of the totals), so there is no
+// scan kernel between the histogram and the scatter.  Inside a block the eight warps own consecutive runs of 256
+// elements: each first counts its digits, the counts are turned into per-warp start offsets (block base + the
+// earlier warps' counts), then every warp ranks its elements in index order.
+// `n_blocks` (the table's row length) is a multiple of 8.
 __global__ void __launch_bounds__(kSortWarps * 32)
 sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restrict__ rows_in,
                     const int32_t* __restrict__ kept, const int32_t* __restrict__ budget_row,
@@ -129,10 +85,44 @@ sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restri
                     int32_t* __restrict__ keys_out, int32_t* __restrict__ rows_out, int n, int cap, int shift,
                     int n_blocks) {
   __shared__ int cnt[kSortWarps][kSortBins];
+  __shared__ int base[kSortBins];                         // row totals, then this block's first position per digit
+  __shared__ int warp_tot[kSortWarps];
+  static_assert(kSortBins == 2 * kSortWarps * 32, "two digits per thread");
   const int g = blockIdx.y, blk = blockIdx.x, warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int S_layer = min(budget_row[0], cap);
   if (!sort_pass_needed(S_layer, shift)) return;
   if (blk * kSortBlockItems >= n) return;                 // uniform over the block
+  // ---- this block's base per digit, from the raw digit table (thread t owns digits 2t and 2t + 1)
+  const int32_t* tg = table + (size_t)g * kSortBins * n_blocks;
+  int before[2], total[2];
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int4* row = reinterpret_cast<const int4*>(tg + (size_t)(2 * threadIdx.x + u) * n_blocks);
+    int all = 0, pre = 0;
+    for (int v4 = 0; v4 < n_blocks / 4; ++v4) {
+      const int4 x = row[v4];
+      const int b0 = 4 * v4;
+      all += x.x + x.y + x.z + x.w;
+      pre += (b0 < blk ? x.x : 0) + (b0 + 1 < blk ? x.y : 0) + (b0 + 2 < blk ? x.z : 0) + (b0 + 3 < blk ? x.w : 0);
+    }
+    total[u] = all;
+    before[u] = pre;
+  }
+  {
+    const int mine = total[0] + total[1];
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int lower = incl - mine;                               // digits below this thread's, all blocks
+    for (int w = 0; w < warp; ++w) lower += warp_tot[w];
+    base[2 * threadIdx.x] = lower + before[0];
+    base[2 * threadIdx.x + 1] = lower + total[0] + before[1];
+  }
   const int32_t* kg = keys_in + (size_t)g * n;
   const int32_t* rg = rows_in + (size_t)g * n;
   const int32_t* kept_g = kept + (size_t)g * cap;
@@ -150,9 +140,8 @@ sort_scatter_kernel(const int32_t* __restrict__ keys_in, const int32_t* __restri
     if (key[r] >= 0) atomicAdd(&cnt[warp][(key[r] >> shift) & (kSortBins - 1)], 1);
   }
   __syncthreads();
-  const int32_t* tg = table + (size_t)g * kSortBins * n_blocks;
   for (int b = threadIdx.x; b < kSortBins; b += blockDim.x) {
-    int run = tg[(size_t)b * n_blocks + blk];
+    int run = base[b];
 #pragma unroll
     for (int w = 0; w < kSortWarps; ++w) {
       const int c = cnt[w][b];

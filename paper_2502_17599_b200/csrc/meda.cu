@@ -590,11 +590,6 @@ meda_status launch_group_reduce(meda_ctx* ctx, const void* k, const void* v, con
       }
       {
         LaunchScope scope(ctx, MEDA_K_GROUP, st);
-        sort_scan_kernel<<<c.n_kv_heads, 1024, 0, st>>>(ctx->ws.sort_table, kSortBins * ctx->sort_chunks, budget_row,
-                                                        cap, shift);
-      }
-      {
-        LaunchScope scope(ctx, MEDA_K_GROUP, st);
         sort_scatter_kernel<<<grid, kSortWarps * 32, 0, st>>>(keys, rows, idx_conserved, budget_row,
                                                               ctx->ws.sort_table, ko, ro, n, cap, shift,
                                                               ctx->sort_chunks);
@@ -895,7 +890,7 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
   }
   if (st == MEDA_OK) st = carve(&ws.ent_partial, ctx->ent_slots, &ws.bytes);
   if (st == MEDA_OK) st = carve(&ws.decode_partial, (int64_t)c.n_q_heads * kDecSplits * (c.head_dim + 2), &ws.bytes);
-  ctx->sort_chunks = (int)((n + kSortBlockItems - 1) / kSortBlockItems + 7) / 8 * 8;   // padded: the scan works on whole vectors
+  ctx->sort_chunks = (int)((n + kSortBlockItems - 1) / kSortBlockItems + 7) / 8 * 8;   // padded: the scatter reads whole vectors
   ctx->seg_chunks = (int)((n + kSegChunk - 1) / kSegChunk);
   ctx->sort_passes = n <= kSortBins ? 1 : (n <= (int64_t)kSortBins * kSortBins ? 2 : 3);
   for (int i = 0; i < 2; ++i) {

@@ -22,7 +22,8 @@
 //    exponent added as an integer; relative error 2.4e-7, the special-function unit's own is 1.7e-7).  That paid
 //    with two epilogue warps per scheduler (a quarter of the exponentials: 5 %); with four the sweep is short of
 //    issue slots rather than of exponentials and the share is zero (a quarter: +4 % time, half: +12 %).
-//  * The two warps that share a row add their states through shared memory at the end of an item.  The
+//  * The two warps that share a row add their states through shared memory at the end of an item (they meet on
+//    an mbarrier with a bounded wait, like every other hand-over here).  The
 //    partial normalisers of an item go to global memory, run-major; the pair of warps that completes a set of 32
 //    rows over all key runs (counted with one atomic per pair and item) merges them, each warp half of the
 //    runs, in run order, and writes the rows' final normalisers together with the per-column constants the
@@ -66,7 +67,7 @@ struct WinStatsParams {
 struct WinStatsSmem {
   static constexpr uint32_t b_off = 0;
   static constexpr uint32_t bar_off = b_off + kWsStages * kWsStageBytes;
-  static constexpr uint32_t n_bars = 2 * kWsStages + 2 * kWsSlots + 2;
+  static constexpr uint32_t n_bars = 2 * kWsStages + 2 * kWsSlots + 2 + 8;     // + one per pair of warps sharing 32 rows
   static constexpr uint32_t misc_off = bar_off + n_bars * 8;
   static constexpr uint32_t pair_off = misc_off + 16;                  // row states handed from a warp to its partner
   static constexpr uint32_t total = pair_off + 8 * 32 * 16 + 8 * 4;
@@ -304,6 +305,7 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
   uint64_t* s_empty = s_full + kWsSlots;
   uint64_t* a_ready = s_empty + kWsSlots;       // the item's query rows are in tensor memory
   uint64_t* a_free = a_ready + 1;               // the item's UMMAs are done with them
+  uint64_t* pair_bar = a_free + 1;              // [8]: the two warps that share 32 rows meet here (bounded waits)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + SH::misc_off);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SH::misc_off + 4);
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -313,6 +315,7 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
     for (uint32_t s = 0; s < kWsSlots; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, kWsEpilogueWarps / 2); }
     mbar_init(a_ready, kWsEpilogueWarps);
     mbar_init(a_free, 1);
+    for (int s = 0; s < 8; ++s) mbar_init(pair_bar + s, 2);
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -393,7 +396,17 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
     const int row_in_block = t * 128 + quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     WinStatsRow row;
-    uint32_t unit_base = 0, item = 0;
+    uint32_t unit_base = 0, item = 0, pair_uses = 0;
+    // The two warps of a pair meet (and see each other's shared-memory writes) through an mbarrier, not a named
+    // barrier: like every other wait of the kernel this one gives up when the block is being aborted, so a warp
+    // whose partner has left the loop after a failed wait does not wait for it for ever.
+    auto pair_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pair_bar + set);
+      bool good = mbar_wait(pair_bar + set, pair_uses & 1u, abort_flag);
+      ++pair_uses;
+      return __all_sync(0xffffffffu, good);
+    };
     WinStatsItem it;
     bool ok = true;
     for (int i = 0; ok && win_stats_item(p, i, it); ++i, ++item) {
@@ -468,11 +481,12 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
       if (!ok) break;
       unit_base += (uint32_t)(it.n_tiles * it.m_tiles);
 
-      // ---- the two halves of a row meet in the half-0 warp (through shared memory, a 64-thread barrier per set)
+      // ---- the two halves of a row meet in the half-0 warp (through shared memory)
       float4* pair_state = reinterpret_cast<float4*>(smem + SH::pair_off) + set * 32 + lane;
       volatile int* pair_flag = reinterpret_cast<volatile int*>(smem + SH::pair_off + 8 * 32 * 16) + set;
       if (half == 1) *pair_state = make_float4(row.mv, row.zv, row.mt, row.zt);
-      asm volatile("bar.sync %0, 64;" ::"r"(1 + set) : "memory");
+      ok = pair_sync();
+      if (!ok) break;
       if (half == 0) {
         const float4 o = *pair_state;
         merge_mz2(row.mv, row.zv, o.x, o.y);
@@ -499,7 +513,8 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
         last = ticket == (unsigned int)p.chunks - 1u;      // every key run of these rows has been written
         if (lane == 0) *pair_flag = last ? 1 : 0;
       }
-      asm volatile("bar.sync %0, 64;" ::"r"(1 + set) : "memory");
+      ok = pair_sync();
+      if (!ok) break;
       last = *pair_flag != 0;                              // uniform over the pair of warps
       if (last) {
         // each warp of the pair merges half of the key runs, the half-0 warp joins the halves and writes the row
@@ -508,7 +523,8 @@ window_stats_kernel(const __grid_constant__ CUtensorMap map_k, const WinStatsPar
         float4 mine4 = make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
         if (valid) mine4 = win_stats_merge_runs(my_part, rows_total, half ? c_mid : 0, half ? p.chunks : c_mid);
         if (half == 1) *pair_state = mine4;
-        asm volatile("bar.sync %0, 64;" ::"r"(1 + set) : "memory");
+        ok = pair_sync();
+        if (!ok) break;
         if (half == 0) {
           if (valid) {
             const float4 o = *pair_state;

@@ -38,7 +38,7 @@ class CompressionPass:
         self.device = device
         # Layers are independent inside each phase, so they alternate between `n_streams` streams, each
         # with its own context (scratch memory): the short, latency-bound kernels of one layer
-        # (selection, sort passes, scans, reductions of partials) then run beside the long kernels of
+        # (selection, sort passes, reductions of partials) then run beside the long kernels of
         # the next instead of leaving the GPU idle.
         self.contexts = [binding.Context.for_workload(wl, **ctx_overrides) for _ in range(max(1, n_streams))]
         self.ctx = self.contexts[0]

@@ -19,6 +19,16 @@ def _built():
     build.build()
 
 
+def _alternating_spans(n_text, n_visual, repeats, tail_text):
+    """((begin, end, modality), ...): `repeats` times (text, visual), then a text tail."""
+    spans, at = [], 0
+    for _ in range(repeats):
+        spans.append((at, at + n_text, 0)); at += n_text
+        spans.append((at, at + n_visual, 1)); at += n_visual
+    spans.append((at, at + tail_text, 0))
+    return tuple(spans)
+
+
 def small_cases():
     return [
         W.WORKLOADS["tiny"],
@@ -33,6 +43,10 @@ def small_cases():
         W.small_variant("tc_w32_g5", window=32, n_q_heads=10, n_kv_heads=2, seed=6,
                         spans=((0, 37, 0), (37, 37 + 9 * 61, 1), (37 + 9 * 61, 37 + 9 * 61 + 40, 0))),   # n = 626 = 2 x 256 + 114
         W.small_variant("tc_w32_g8", window=32, n_q_heads=16, n_kv_heads=2, seed=7),
+        # 224 query rows per KV head (the long-video shape) over short alternating spans: every 32-key chunk holds
+        # both modalities, so the normaliser sweep takes its mixed-modality path everywhere
+        W.small_variant("tc_w32_g7_alternating", window=32, n_q_heads=14, n_kv_heads=2, seed=9, frame_tokens=0,
+                        spans=_alternating_spans(13, 18, 21, 40)),
         W.WORKLOADS["long_video_19k"].with_(name="long_video_19k_2l", n_layers=2),
     ]
 

@@ -128,7 +128,9 @@ select_topk_kernel(const float* __restrict__ scores, const uint8_t* __restrict__
 // ---------------------------------------------------------------------------------------------
 constexpr int kSelMaxClusterSize = 8;
 constexpr int kSelBins = 2048;                    // 11-bit digits: 11 + 11 + 10 bits of the score key
-constexpr int kSelPerThread = 4;                  // consecutive tokens per thread in the compaction
+constexpr int kSelPerThread = 16;                 // consecutive tokens per thread and round of the compaction
+constexpr int kSelBlockStep = 4096;               // a block's share of the tokens is a multiple of this
+constexpr int kSelMaxRounds = 4;                  // compaction rounds per block: 64K tokens, more than shared memory holds
 
 struct SelectClusterSmem {
   int chunk;          // tokens per block
@@ -136,12 +138,12 @@ struct SelectClusterSmem {
 };
 __host__ __device__ inline SelectClusterSmem select_cluster_smem(int n, int cluster_size) {
   SelectClusterSmem L;
-  const int step = kSelThreads * kSelPerThread;
+  const int step = kSelBlockStep;
   L.chunk = ((n + cluster_size - 1) / cluster_size + step - 1) / step * step;
   int off = 0;
   L.keys_off = off;  off += L.chunk * 4;
-  L.hist_off = off;  off += kSelBins * 4;
-  L.total_off = off; off += kSelBins * 4;
+  L.hist_off = off;  off += 2 * kSelBins * 4;     // two histograms, used by alternate radix passes
+  L.total_off = off;
   L.misc_off = off;  off += 256;
   L.total = off;
   return L;
@@ -180,14 +182,14 @@ __device__ __forceinline__ int block_exclusive_sum(int v, int* scratch, int& tot
 inline int select_cluster_size(int n, int n_heads, int sm_count, int smem_limit) {
   if (select_cluster_smem(n, kSelMaxClusterSize).total > smem_limit) return 0;
   int c = kSelMaxClusterSize;
-  while (c > 1 && ((n + c - 1) / c < kSelThreads * kSelPerThread || n_heads * c > sm_count) &&
+  while (c > 1 && ((n + c - 1) / c < kSelBlockStep || n_heads * c > sm_count) &&
          select_cluster_smem(n, c / 2).total <= smem_limit)
     c /= 2;
   return c;
 }
 
 template <int kSelClusterSize>
-__global__ void __cluster_dims__(kSelClusterSize, 1, 1) __launch_bounds__(kSelThreads)
+__global__ void __cluster_dims__(kSelClusterSize, 1, 1) __launch_bounds__(kSelThreads, 1)
 select_topk_cluster_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ modality,
                            const int32_t* __restrict__ budget_row, int32_t* __restrict__ idx_conserved,
                            int32_t* __restrict__ idx_less, int n, int cap, int* status) {
@@ -197,7 +199,6 @@ select_topk_cluster_kernel(const float* __restrict__ scores, const uint8_t* __re
   const SelectClusterSmem L = select_cluster_smem(n, kSelClusterSize);
   unsigned int* keys = reinterpret_cast<unsigned int*>(sel_smem + L.keys_off);
   unsigned int* hist = reinterpret_cast<unsigned int*>(sel_smem + L.hist_off);
-  unsigned int* total = reinterpret_cast<unsigned int*>(sel_smem + L.total_off);
   int* misc = reinterpret_cast<int*>(sel_smem + L.misc_off);
   // misc: [0..32] scan scratch, [40] text candidates of this block, [41] kept for sure, [42] equal to the
   // threshold, [44] digit, [45] remaining
@@ -240,64 +241,78 @@ select_topk_cluster_kernel(const float* __restrict__ scores, const uint8_t* __re
     for (int pass = 0; pass < 3; ++pass) {
       const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
       const unsigned int bins = pass == 2 ? 1024u : 2048u;
-      for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) hist[b] = 0u;
+      // Alternate passes count into alternate histograms: the other blocks read this block's histogram of pass p
+      // before they arrive at the barrier of pass p + 1, and it is cleared again only in pass p + 2, so one
+      // cluster barrier per pass is enough.
+      unsigned int* h = hist + (pass & 1) * kSelBins;
+      for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) h[b] = 0u;
       __syncthreads();
       for (int j = lo + (int)threadIdx.x; j < min(hi, n_cand); j += kSelThreads) {
         const unsigned int key = keys[j - lo];
-        if (modality[j] == cls && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & (bins - 1u)], 1u);
+        if (modality[j] == cls && (key & mask) == prefix) atomicAdd(&h[(key >> shift) & (bins - 1u)], 1u);
       }
       cluster.sync();                                   // every block's histogram is complete
-      for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) {
-        unsigned int t = 0u;
+      // Thread t owns the bins bins - 1 - 2t and bins - 2 - 2t (from the top down), summed over the cluster; an
+      // exclusive sum over the threads gives the number of keys in all bins above, and the one thread whose bins
+      // hold the `remaining`-th key from the top records the digit.
+      const int b0 = (int)bins - 1 - 2 * (int)threadIdx.x, b1 = b0 - 1;       // b1 is even: one 8-byte load for both
+      int c0 = 0, c1 = 0;
+      if (b1 >= 0) {
 #pragma unroll
-        for (int r = 0; r < kSelClusterSize; ++r) t += cluster.map_shared_rank(hist, r)[b];
-        total[b] = t;
+        for (int r = 0; r < kSelClusterSize; ++r) {
+          const uint2 pair = *reinterpret_cast<const uint2*>(cluster.map_shared_rank(h, r) + b1);
+          c1 += (int)pair.x;
+          c0 += (int)pair.y;
+        }
       }
-      cluster.sync();                                   // remote reads are done before the histograms are reused
-      if (threadIdx.x < 32) {
-        // lane l owns bins [64 l, 64 l + 64); walk from the top bin down
-        const int lane = threadIdx.x;
-        int mine = 0;
-        for (int b = 0; b < 64; ++b) mine += (int)total[lane * 64 + b];
-        int above = 0;                                  // keys in bins owned by higher lanes
-        for (int o = 31; o > 0; --o) {
-          int y = __shfl_sync(0xffffffffu, mine, o);
-          if (o > lane) above += y;
-        }
-        if (above < remaining && above + mine >= remaining) {
-          int cum = above;
-          for (int b = 63; b >= 0; --b) {
-            const int c = (int)total[lane * 64 + b];
-            if (cum + c >= remaining) { misc[44] = lane * 64 + b; misc[45] = remaining - cum; break; }
-            cum += c;
-          }
-        }
+      int all_keys;
+      const int above = block_exclusive_sum(c0 + c1, misc, all_keys);
+      if (above < remaining && above + c0 + c1 >= remaining) {
+        if (above + c0 >= remaining) { misc[44] = b0; misc[45] = remaining - above; }
+        else { misc[44] = b1; misc[45] = remaining - above - c0; }
       }
       __syncthreads();
       prefix |= (unsigned int)misc[44] << shift;
       mask |= (bins - 1u) << shift;
       remaining = misc[45];
-      __syncthreads();
     }
   }
   const unsigned int threshold = prefix;
   const int take_equal = N > 0 ? remaining : 0;
 
-  // ---- classify own tokens: 2 = kept for sure, 1 = equal to the threshold, 0 = dropped
-  auto classify = [&](int j) -> int {
-    if (j >= n) return 0;
-    if (j >= n_cand) return 2;
-    if (N == 0) return 0;
-    const int md = modality[j];
-    if (md != cls) return (cls == MEDA_VISUAL) ? 2 : 0;
-    const unsigned int key = keys[j - lo];
-    return key > threshold ? 2 : (key == threshold ? 1 : 0);
-  };
+  // ---- classify own tokens, 16 consecutive ones per thread and round: 2 = kept for sure, 1 = equal to the
+  // threshold, 0 = dropped; two bits per token, kept in registers for the compaction below
+  uint32_t codes[kSelMaxRounds];
   int sure = 0, equal = 0;
-  for (int j = lo + (int)threadIdx.x; j < hi; j += kSelThreads) {
-    const int c = classify(j);
-    sure += c == 2;
-    equal += c == 1;
+#pragma unroll
+  for (int r = 0; r < kSelMaxRounds; ++r) {
+    codes[r] = 0u;
+    const int j0 = lo + (r * kSelThreads + (int)threadIdx.x) * kSelPerThread;
+    if (j0 < hi) {
+      // the modality map is padded past n and j0 is a multiple of 16: one 16-byte load; keys: four
+      const uint4 mv = *reinterpret_cast<const uint4*>(modality + j0);
+      const uint32_t mw[4] = {mv.x, mv.y, mv.z, mv.w};
+      const uint4* kp = reinterpret_cast<const uint4*>(keys + (j0 - lo));
+#pragma unroll
+      for (int w4 = 0; w4 < 4; ++w4) {
+        const uint4 kv = kp[w4];
+        const unsigned int kk[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int x = 4 * w4 + b, j = j0 + x;
+          const int md = (int)((mw[w4] >> (8 * b)) & 0xffu);
+          int c;
+          if (j >= n) c = 0;
+          else if (j >= n_cand) c = 2;
+          else if (N == 0) c = 0;
+          else if (md != cls) c = (cls == MEDA_VISUAL) ? 2 : 0;
+          else c = kk[b] > threshold ? 2 : (kk[b] == threshold ? 1 : 0);
+          codes[r] |= (uint32_t)c << (2 * x);
+          sure += c == 2;
+          equal += c == 1;
+        }
+      }
+    }
   }
   sure = __reduce_add_sync(0xffffffffu, sure);
   equal = __reduce_add_sync(0xffffffffu, equal);
@@ -312,37 +327,52 @@ select_topk_cluster_kernel(const float* __restrict__ scores, const uint8_t* __re
     kept_before += m[41] + min(max(take_equal - equal_before, 0), e);
     equal_before += e;
   }
-  cluster.sync();                                       // nobody reads this block's counters after this point
 
-  // ---- ordered compaction of own tokens, kSelPerThread consecutive tokens per thread
-  for (int base = lo; base < hi; base += kSelThreads * kSelPerThread) {
-    const int j0 = base + (int)threadIdx.x * kSelPerThread;
-    int c[kSelPerThread];
-    int eq = 0;
+  // ---- ordered compaction of own tokens.  The positions are computed per thread (16 consecutive tokens), but
+  // written to global memory by the whole block from shared memory, where the sort keys are no longer needed:
+  // kept indices from the front of the buffer, dropped ones from its back (a block's dropped tokens are
+  // contiguous in the less-important list too), so that every global store is a full line.
+  int* stage = reinterpret_cast<int*>(keys);
 #pragma unroll
-    for (int x = 0; x < kSelPerThread; ++x) { c[x] = (j0 + x < hi) ? classify(j0 + x) : 0; eq += c[x] == 1; }
+  for (int r = 0; r < kSelMaxRounds; ++r) {
+    const int r_lo = lo + r * kSelThreads * kSelPerThread;             // first token of the round
+    if (r_lo >= hi) break;                                            // uniform over the block
+    const int r_n = min(kSelThreads * kSelPerThread, hi - r_lo);       // tokens of the round
+    const int j0 = r_lo + (int)threadIdx.x * kSelPerThread;
+    const uint32_t cd = codes[r];
+    // tokens equal to the threshold: code 1; kept for sure: code 2
+    const uint32_t eq_bits = cd & ~(cd >> 1) & 0x55555555u, sure_bits = (cd >> 1) & 0x55555555u;
     int eq_total, keep_total;
-    int eq_rank = equal_before + block_exclusive_sum(eq, misc, eq_total);
-    int keep = 0;
-    bool k[kSelPerThread];
+    int eq_rank = equal_before + block_exclusive_sum(__popc(eq_bits), misc, eq_total);
+    uint32_t keep_bits = sure_bits;
 #pragma unroll
     for (int x = 0; x < kSelPerThread; ++x) {
-      k[x] = c[x] == 2 || (c[x] == 1 && eq_rank < take_equal);
-      eq_rank += c[x] == 1;
-      keep += k[x];
+      if ((eq_bits >> (2 * x)) & 1u) {
+        if (eq_rank < take_equal) keep_bits |= 1u << (2 * x);
+        ++eq_rank;
+      }
     }
-    int pos = kept_before + block_exclusive_sum(keep, misc, keep_total);
+    // (the first barrier inside the sum above also orders the last reads of the keys before the stores below)
+    int pos = block_exclusive_sum(__popc(keep_bits), misc, keep_total);   // kept tokens of the round before mine
 #pragma unroll
     for (int x = 0; x < kSelPerThread; ++x) {
       const int j = j0 + x;
       if (j < hi) {
-        if (k[x]) { out_c[pos] = j; ++pos; }
-        else out_l[j - pos] = j;
+        if ((keep_bits >> (2 * x)) & 1u) { stage[pos] = j; ++pos; }
+        else stage[r_n - 1 - ((j - r_lo) - pos)] = j;
       }
     }
+    __syncthreads();
+    const int drop_total = r_n - keep_total;
+    int32_t* dst_c = out_c + kept_before;
+    int32_t* dst_l = out_l + (r_lo - kept_before);
+    for (int e = threadIdx.x; e < keep_total; e += kSelThreads) dst_c[e] = stage[e];
+    for (int e = threadIdx.x; e < drop_total; e += kSelThreads) dst_l[e] = stage[r_n - 1 - e];
     kept_before += keep_total;
     equal_before += eq_total;
+    __syncthreads();                                                  // the buffer is reused by the next round
   }
+  cluster.sync();                                       // no block leaves while another may still read its counters
 }
 
 }  // namespace meda

@@ -417,6 +417,35 @@ def test_select_beyond_cluster_capacity_uses_the_single_block_kernel():
     ctx.close()
 
 
+@pytest.mark.parametrize("n", [150_001, 300_017])
+def test_select_with_several_compaction_rounds_per_block(n):
+    """Between 131,072 and 393,216 tokens a block of the selection cluster owns more tokens than one compaction
+    round takes (16 per thread): two rounds at 150K, three at 300K, the last one ragged.  Same ranking and
+    tie-break as everywhere, with a run of exact ties that straddles a round's border."""
+    wl = W.small_variant(f"select_{n}", dtype="f32", n_layers=1, n_q_heads=1, n_kv_heads=1, head_dim=64, window=8,
+                         spans=((0, 1000, 0), (1000, n - 500, 1), (n - 500, n, 0)), rho=0.1, frame_tokens=0)
+    ctx = make_ctx(wl)
+    rng = np.random.default_rng(6)
+    a_s = rng.random(n).astype(np.float32)
+    a_s[16_300:16_500] = a_s[16_300]                # exact ties across the first round's border of block 0
+    mod = wl.modality().numpy()
+    scores = torch.from_numpy(a_s[None]).cuda()
+    idx_c = torch.full((1, n), -1, dtype=torch.int32, device="cuda")
+    idx_l = torch.full((1, n), -1, dtype=torch.int32, device="cuda")
+    # third budget: every text candidate, every visual candidate above the tied score and 100 of the 200 tied ones
+    # (the lowest indices), so that the threshold falls inside the run of ties
+    above = int((a_s[1000: n - 3000] > a_s[16_300]).sum())
+    for M, N in ((3000, 1040), (10, 2000), (3000, 1000 + above + 100)):
+        budgets = torch.tensor([[M + N, M, N]], dtype=torch.int32, device="cuda")
+        ctx.select_topk(0, scores, budgets, idx_c, idx_l, n)
+        ctx.check()
+        assert P.compare_selection(idx_c[0, : M + N].cpu().numpy(), a_s.astype(np.float64), mod, M, N) == 0
+        less = idx_l[0, : n - M - N].cpu().numpy()
+        assert (np.diff(less) > 0).all() and less.size + M + N == n
+        assert np.intersect1d(less, idx_c[0, : M + N].cpu().numpy()).size == 0
+    ctx.close()
+
+
 @pytest.mark.parametrize("wl", [
     W.small_variant(),                                                          # CUDA-core kernels for both terms
     W.small_variant("evt_tc_w32", window=32, seed=4),                           # E_TV on the tensor cores, E_VT on CUDA cores

@@ -78,8 +78,9 @@ typedef struct {
 /* Creates a context: validates the configuration, uploads the modality map built from
  * `spans_host` (host memory, n_spans entries) and allocates all scratch memory on the current
  * device (the only allocating call).  Supported shapes: head_dim in {64, 128, 256} for fp32 and
- * bf16, n_q_heads a multiple of n_kv_heads, 1 <= window <= min(n_tokens, 128), n_layers <= 1024.
- * On failure *out is NULL and the status says why. */
+ * bf16, n_q_heads a multiple of n_kv_heads, 1 <= window <= min(n_tokens, 128), n_layers <= 1024; one head's
+ * cache below 4 GiB (n_tokens * head_dim * element size < 2^32) and n_tokens * n_kv_heads < 2^31 (MEDA_ERR_SHAPE
+ * otherwise).  On failure *out is NULL and the status says why. */
 meda_status meda_create(const meda_config* config, const meda_span* spans_host, int32_t n_spans, meda_ctx** out);
 
 /* Frees the context's scratch memory.  The caller must have synchronised the streams that used it. */

@@ -787,6 +787,10 @@ meda_status meda_create(const meda_config* config, const meda_span* spans_host, 
       c.window > kMaxWindow)
     return MEDA_ERR_SHAPE;
   if (c.head_dim != 64 && c.head_dim != 128 && c.head_dim != 256) return MEDA_ERR_SHAPE;
+  // byte offsets of a row inside one head's cache are 32-bit in the segmented average, token indices int32 everywhere
+  if ((int64_t)c.n_tokens * c.head_dim * (c.dtype == MEDA_F32 ? 4 : 2) >= (int64_t(1) << 32) ||
+      (int64_t)c.n_tokens * c.n_kv_heads >= (int64_t(1) << 31))
+    return MEDA_ERR_SHAPE;
   if (c.beta_recent < 0 || c.beta_important < 0 || c.beta_recent + c.beta_important <= 0) return MEDA_ERR_INVALID_ARG;
   if (c.min_budget < 1 || c.min_budget > c.n_tokens) return MEDA_ERR_BUDGET_INFEASIBLE;
   if (c.global_budget < (int64_t)c.n_layers * c.min_budget || c.global_budget > (int64_t)c.n_layers * c.n_tokens)

@@ -57,6 +57,9 @@ def test_create_rejects_bad_arguments_before_touching_the_device(lib):
     assert status_of(head_dim=96) == B.MEDA_ERR_SHAPE
     assert status_of(window=101) == B.MEDA_ERR_SHAPE
     assert status_of(window=200, n_tokens=1000, spans=((0, 1000, 1),), global_budget=500) == B.MEDA_ERR_SHAPE
+    # one head's cache of 4 GiB or more (32-bit byte offsets inside a head): 2^24 tokens x 256 dims x 4 bytes
+    assert status_of(n_tokens=1 << 24, head_dim=256, dtype="f32", spans=((0, 1 << 24, 1),),
+                     global_budget=1 << 20) == B.MEDA_ERR_SHAPE
     assert status_of(global_budget=3) == B.MEDA_ERR_BUDGET_INFEASIBLE
     assert status_of(global_budget=201) == B.MEDA_ERR_BUDGET_INFEASIBLE
     assert status_of(spans=((0, 10, 0), (11, 100, 1))) == B.MEDA_ERR_INVALID_ARG      # gap
